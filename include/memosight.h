@@ -1,0 +1,227 @@
+/*
+ * memosight.h -- C ABI of the MemoSight per-step attention hot path (B200, sm_100a).
+ *
+ * MemoSight inference alternates two things (paper Sec. 2.1, Algorithm 1):
+ *   - Predict+Verify steps: a small block of new tokens -- the pending candidate
+ *     tokens, causal among themselves, followed by d foresight tokens that see
+ *     the prefix and themselves only -- runs one forward pass against the KV
+ *     cache; the greedy rule accepts the longest draft prefix that equals the
+ *     model's own argmax; accepted tokens are appended to the cache;
+ *   - compression: when a reasoning step ends, ceil(n/c) memory tokens and one
+ *     output token are appended behind it and the step's n verbose entries are
+ *     evicted from the KV cache, which therefore stays compacted.
+ * This library implements the attention-side work of that loop, one call per
+ * operation, as CUDA kernels.  There is no CPU fallback: every call other than
+ * the host-only layout helpers fails with MS_ERR_CUDA when no device is usable.
+ *
+ * Conventions that hold for every call unless its comment says otherwise:
+ *   - "device" pointers are device memory owned by the caller, valid until the
+ *     work queued on `stream` has finished; "host" pointers are ordinary host
+ *     memory read or written before the call returns.
+ *   - bf16 tensors are raw 16-bit patterns (the upper half of an IEEE binary32);
+ *     base pointers of bf16 tensors must be 16-byte aligned.
+ *   - calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL is
+ *     the default stream), never synchronise, never allocate device memory and
+ *     never read device scalars on the host: ragged lengths stay on the device
+ *     and the caller supplies host-side upper bounds for launch sizing.
+ *   - return value: MS_OK or a negative MS_ERR_* code.  Arguments are validated
+ *     on the host before anything is launched; a rejected call has no effect.
+ *     Device code never traps; the only device-side failure (a bounded wait that
+ *     ran out) is recorded in the workspace and read by memosight_attn_status().
+ *   - GQA: query head h reads KV head h / (n_q_heads / n_kv_heads).
+ */
+#ifndef MEMOSIGHT_H_
+#define MEMOSIGHT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define MS_OK 0
+#define MS_ERR_INVALID_ARG (-1)         /* null pointer, negative size, inconsistent sizes        */
+#define MS_ERR_UNSUPPORTED_SHAPE (-2)   /* a size outside the documented limits                   */
+#define MS_ERR_WORKSPACE_TOO_SMALL (-3) /* workspace_bytes below the *_workspace_bytes() answer   */
+#define MS_ERR_ALIGNMENT (-4)           /* a pointer or stride breaks the 16-byte rule            */
+#define MS_ERR_CUDA (-5)                /* a CUDA runtime/driver call failed; see last_cuda_error */
+#define MS_ERR_DEVICE_TIMEOUT (-6)      /* a bounded device-side wait ran out (attn_status only)  */
+
+typedef void* memosight_stream_t; /* a cudaStream_t */
+
+#if defined(__GNUC__)
+#define MS_API __attribute__((visibility("default")))
+#else
+#define MS_API
+#endif
+
+/* RoPE flags */
+#define MS_ROPE_NEOX 0u          /* pair (i, i + D/2): rotate-half, the default                  */
+#define MS_ROPE_INTERLEAVED 1u   /* pair (2i, 2i+1)                                              */
+#define MS_POS_HALF_UNITS 2u     /* pos_id counts half positions (exact UPL centres)             */
+
+/* Library version (major*10000 + minor*100 + patch). */
+MS_API int32_t memosight_version(void);
+/* Static, NUL-terminated description of a status code. */
+MS_API const char* memosight_status_string(int32_t status);
+/* The cudaError_t (as int) behind the most recent MS_ERR_CUDA of this thread, 0 if none. */
+MS_API int32_t memosight_last_cuda_error(void);
+
+/* ---- Position layout (host-only integer helpers; Sec. 2.1.2, Sec. 2.2) ------------------- */
+
+/* Adaptive Memory Allocation: number of memory tokens for a step of n tokens at
+ * compression ratio c, l = ceil(n / c).  n >= 0, c >= 1, else MS_ERR_INVALID_ARG. */
+MS_API int32_t memosight_ama(int32_t n, int32_t c);
+
+/* Uniform Position Layout: the step's n tokens hold PIDs rho_first .. rho_first+n-1
+ * and are cut into l = ceil(n/c) sequential groups of c (last may be shorter);
+ * memory token g gets the centre PID of group g.  A half-integer centre (even
+ * group size) is rounded down, or returned exactly in half positions when flags
+ * has MS_POS_HALF_UNITS (value = 2*centre).  pid_out: host, capacity cap >= l.
+ * Returns l, or a negative code (MS_ERR_INVALID_ARG also when cap < l). */
+MS_API int32_t memosight_upl_pids(int32_t rho_first, int32_t n, int32_t c, uint32_t flags,
+                           int32_t* pid_out, int32_t cap);
+
+/* PID of the output token <o> that closes a step: the step's last PID plus one. */
+MS_API int32_t memosight_out_pid(int32_t rho_first, int32_t n);
+
+/* PIDs of one step block (Sec. 2.1.1; Sec. 2.2, foresight tokens): rows 0..n_c-1
+ * are the candidates (p0, p0+1, ...); row n_c+k-1 is foresight token f_k, which
+ * takes the PID just before its prediction target: (PID of the last regular
+ * token it sees) + k.  anchor (host, [d] or NULL): how many candidates f_k sees;
+ * NULL means all n_c.  pid_out: host [n_c + d].  Returns MS_OK or a code. */
+MS_API int32_t memosight_step_pids(int32_t p0, int32_t n_c, int32_t d, const int32_t* anchor,
+                            int32_t* pid_out);
+
+/* ---- RoPE at token-specific position IDs (Sec. 2.1.2, UPL paragraph) --------------------- */
+
+/* Rotates, in place, every head vector of the T new tokens by the token's own PID.
+ *   q       device bf16 [T][H_q][D]   (may be NULL when H_q == 0)
+ *   k       device bf16 [T][H_kv][D]  (may be NULL when H_kv == 0)
+ *   pos_id  device int32 [T]
+ *   inv_freq host double [D/2] or NULL; NULL means theta_i = rope_base^(-2i/D)
+ * Angles and the rotation are evaluated in fp64 and rounded to bf16 once.
+ * D even, 2 <= D <= 256.  T == 0 is a no-op. */
+MS_API int32_t memosight_rope_qk(void* q, void* k, const int32_t* pos_id, int32_t T, int32_t H_q,
+                          int32_t H_kv, int32_t D, double rope_base, const double* inv_freq,
+                          uint32_t flags, memosight_stream_t stream);
+
+/* ---- Step attention (Sec. 2.1.1 masks; Sec. 2.3 "Attention Mask Strategy") --------------- */
+
+/* One layer of attention of all sequences' step blocks against the compacted cache.
+ * Visibility: every one of the kv_len[b] cache entries is visible to every row of
+ * block b (the verbose steps were evicted; prompt, memory, output tokens and the
+ * current step's accepted tokens remain).  Among the block's own n_q keys, key j
+ * is visible to row i iff j == i, or j is a candidate (j < n_cand[b]) and
+ * j < a_i, where a_i = i for a candidate row (causal) and a_i = anchor[row]
+ * (default n_cand[b]) for a foresight row.  Foresight keys are visible to no
+ * other row.  The mask is evaluated from this metadata; no matrix is built. */
+typedef struct memosight_attn_params {
+  uint32_t struct_size;      /* sizeof(memosight_attn_params), for ABI growth                 */
+  int32_t batch;             /* B >= 0                                                         */
+  int32_t n_q_heads;         /* H_q, multiple of n_kv_heads                                    */
+  int32_t n_kv_heads;        /* H_kv                                                           */
+  int32_t head_dim;          /* D: 64 or 128 on the tensor-core path; any multiple of 32 up to
+                                256 on the general path                                        */
+  const void* k_cache;       /* device bf16, one layer: [H_kv][n_slots][D], post-RoPE          */
+  const void* v_cache;       /* device bf16, same layout                                       */
+  int64_t kv_head_stride;    /* elements between KV heads (>= n_slots*D, multiple of 8)        */
+  int64_t n_slots;           /* slots per KV head (< 2^31)                                     */
+  const int64_t* kv_off;     /* device [B]: first slot of sequence b                           */
+  const int32_t* kv_len;     /* device [B]: valid entries L_b (kv_off[b]+L_b <= n_slots)       */
+  int32_t max_kv_len;        /* host upper bound of kv_len[]                                   */
+  int32_t max_nq;            /* host upper bound of the block sizes, 1..16                     */
+  const int32_t* q_off;      /* device [B+1]: rows of block b are q_off[b] .. q_off[b+1]-1     */
+  const int32_t* n_cand;     /* device [B]: candidates in block b (the block's first rows)     */
+  const int32_t* anchor;     /* device [T] or NULL; read only for foresight rows               */
+  int32_t total_rows;        /* T = q_off[B] (host copy)                                       */
+  float sm_scale;            /* softmax scale; 0 means 1/sqrt(D)                               */
+  const void* q;             /* device bf16 [T][H_q][D], post-RoPE                             */
+  const void* k_step;        /* device bf16 [T][H_kv][D], post-RoPE                            */
+  const void* v_step;        /* device bf16 [T][H_kv][D]                                       */
+  void* out;                 /* device bf16 [T][H_q][D]                                        */
+  float* lse;                /* device fp32 [T][H_q], natural-log sum-exp, or NULL             */
+  void* workspace;           /* device scratch, 256-byte aligned                               */
+  size_t workspace_bytes;    /* >= memosight_attn_workspace_bytes(...)                         */
+} memosight_attn_params;
+
+/* Scratch size for memosight_attn_step with these bounds (0 on invalid input).
+ * It does not depend on the cache length: the split-KV partials are per CTA. */
+MS_API size_t memosight_attn_workspace_bytes(int32_t batch, int32_t n_q_heads, int32_t n_kv_heads,
+                                      int32_t head_dim, int32_t max_kv_len, int32_t max_nq);
+
+/* Queues the attention of one layer (split-KV pass + log-sum-exp merge).
+ * Limits: n_q_heads/n_kv_heads <= 16; max_nq <= 16; batch <= 8192 per call.
+ * Blocks with max_nq * (H_q/H_kv) <= 64 and D in {64,128} take the tensor-core
+ * path; anything else inside the limits takes the slower general path.
+ * The workspace may be reused by the next call on the same stream; two calls
+ * that overlap on the GPU need two workspaces. */
+MS_API int32_t memosight_attn_step(const memosight_attn_params* params, memosight_stream_t stream);
+
+/* Synchronises `stream` and returns MS_OK, or MS_ERR_DEVICE_TIMEOUT if a kernel
+ * of the last memosight_attn_step on this workspace gave up on a bounded wait
+ * (its output is then undefined).  Meant for tests and debugging. */
+MS_API int32_t memosight_attn_status(const void* workspace, memosight_stream_t stream);
+
+/* ---- KV compaction and append (Sec. 2.1.2; Algorithm 1: UpdateCache, S <- S (+) A) ------- */
+
+/* Evicts one verbose step per sequence from every layer's K and V cache, in place:
+ * entries seg_start[b] .. seg_start[b]+seg_len[b]-1 are dropped and everything
+ * behind them (the memory tokens and <o> appended after the step, and anything
+ * later) moves up, order and bits preserved:  new = old[0:s) ++ old[s+n:L).
+ *   k_cache, v_cache  device bf16 [n_layers][H_kv][n_slots][D]; layer_stride and
+ *                     kv_head_stride in elements (multiples of 8)
+ *   kv_off            device int64 [B]
+ *   kv_len            device int32 [B], in/out: becomes L - n
+ *   seg_start,seg_len device int32 [B]; seg_len[b] == 0 skips sequence b; a segment
+ *                     that does not fit in [0, L) is ignored (sequence untouched)
+ *   src_idx           device int32 [B][idx_stride] or NULL: old index of each new
+ *                     entry (first L-n values of row b are written)
+ *   max_tail          host upper bound of L - s - n (entries that move)
+ * D*2 bytes must be a multiple of 16. */
+MS_API int32_t memosight_kv_compact(void* k_cache, void* v_cache, int32_t n_layers, int64_t layer_stride,
+                             int64_t kv_head_stride, int32_t batch, int32_t n_kv_heads,
+                             int32_t head_dim, const int64_t* kv_off, int32_t* kv_len,
+                             const int32_t* seg_start, const int32_t* seg_len, int32_t* src_idx,
+                             int32_t idx_stride, int32_t max_tail, memosight_stream_t stream);
+
+/* Appends the accepted candidates of each block to one layer's cache: the first
+ * n_keep[b] rows of block b in k_step/v_step go to slots kv_len[b] .. of sequence
+ * b.  n_keep[b] is clamped to [0, n_cand[b]]: a foresight row is never cached
+ * (no later token may attend to it, Sec. 2.3).  kv_len[b] += n_keep[b] iff
+ * bump_len != 0 (pass it on the last layer).  max_nq: host bound of block sizes.
+ *   k_cache, v_cache device bf16 [H_kv][n_slots][D]; k_step, v_step device bf16 [T][H_kv][D] */
+MS_API int32_t memosight_kv_append(void* k_cache, void* v_cache, int64_t kv_head_stride, int32_t batch,
+                            int32_t n_kv_heads, int32_t head_dim, const int64_t* kv_off,
+                            int32_t* kv_len, const void* k_step, const void* v_step,
+                            const int32_t* q_off, const int32_t* n_cand, const int32_t* n_keep,
+                            int32_t max_nq, int32_t bump_len, memosight_stream_t stream);
+
+/* ---- Greedy accept (Sec. 2.1.1 and its footnote) ----------------------------------------- */
+
+/* Scratch size for memosight_accept (0 on invalid input). */
+MS_API size_t memosight_accept_workspace_bytes(int32_t total_rows, int32_t vocab);
+
+/* Row argmax of fp32 logits and, per sequence, the length of the longest draft
+ * prefix that equals the argmax row by row.
+ *   logits     device fp32 [T][ld_v] (ld_v >= V; 16-byte aligned rows read faster)
+ *   row_off    device int32 [B+1]; rows of sequence b: row_off[b] .. row_off[b+1]-1
+ *   draft      device int32 [T]: the token row r's prediction must equal, or -1
+ *              where nothing is to be verified (last candidate row, foresight rows)
+ *   argmax_out device int32 [T]: lowest index of the row maximum; a NaN counts as
+ *              larger than any number and the first NaN wins
+ *   n_match    device int32 [B]: largest m with draft >= 0 and argmax == draft on
+ *              the block's rows 0..m-1
+ * Row convention: row i of a block holds candidate c_i and predicts the token
+ * after it, so draft[i] = c_{i+1}; tokens c_0..c_{n_match} become permanent and
+ * argmax_out[row n_match] is the next token. */
+MS_API int32_t memosight_accept(const float* logits, int64_t ld_v, int32_t vocab, const int32_t* row_off,
+                         int32_t batch, int32_t total_rows, const int32_t* draft,
+                         int32_t* argmax_out, int32_t* n_match, void* workspace,
+                         size_t workspace_bytes, memosight_stream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MEMOSIGHT_H_ */

@@ -1,0 +1,235 @@
+"""Thin ctypes binding of libmemosight.so: same names as the C ABI, argument
+marshalling only.  Every step of the path runs in the CUDA kernels behind the
+library; there is no CPU fallback -- if the library is missing or a call fails,
+an exception is raised.
+
+Tensor arguments may be torch tensors (their ``data_ptr()`` is passed; they must
+be contiguous and on the current CUDA device), ``None`` for an optional pointer,
+or plain integers that already are addresses.  Host-side arrays are numpy arrays
+or Python lists.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+
+from . import build as _build
+
+MS_OK = 0
+MS_ERR_INVALID_ARG = -1
+MS_ERR_UNSUPPORTED_SHAPE = -2
+MS_ERR_WORKSPACE_TOO_SMALL = -3
+MS_ERR_ALIGNMENT = -4
+MS_ERR_CUDA = -5
+MS_ERR_DEVICE_TIMEOUT = -6
+
+MS_ROPE_NEOX = 0
+MS_ROPE_INTERLEAVED = 1
+MS_POS_HALF_UNITS = 2
+
+
+class MemosightError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        msg = lib().memosight_status_string(status).decode()
+        extra = ""
+        if status == MS_ERR_CUDA:
+            extra = f" (cudaError {lib().memosight_last_cuda_error()})"
+        super().__init__(f"{what}: {msg}{extra} [{status}]")
+
+
+class AttnParams(C.Structure):
+    """Mirror of ``memosight_attn_params`` (include/memosight.h)."""
+    _fields_ = [
+        ("struct_size", C.c_uint32), ("batch", C.c_int32), ("n_q_heads", C.c_int32),
+        ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32),
+        ("k_cache", C.c_void_p), ("v_cache", C.c_void_p),
+        ("kv_head_stride", C.c_int64), ("n_slots", C.c_int64),
+        ("kv_off", C.c_void_p), ("kv_len", C.c_void_p),
+        ("max_kv_len", C.c_int32), ("max_nq", C.c_int32),
+        ("q_off", C.c_void_p), ("n_cand", C.c_void_p), ("anchor", C.c_void_p),
+        ("total_rows", C.c_int32), ("sm_scale", C.c_float),
+        ("q", C.c_void_p), ("k_step", C.c_void_p), ("v_step", C.c_void_p),
+        ("out", C.c_void_p), ("lse", C.c_void_p),
+        ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+    ]
+
+
+_lib: Optional[C.CDLL] = None
+
+
+def lib() -> C.CDLL:
+    """Loads (building first if a source is newer) the CUDA library; raises if impossible."""
+    global _lib
+    if _lib is None:
+        path = _build.LIB
+        if not os.path.exists(path) or _build.is_stale():
+            path = _build.build()
+        L = C.CDLL(path)
+        L.memosight_status_string.restype = C.c_char_p
+        L.memosight_status_string.argtypes = [C.c_int32]
+        L.memosight_version.restype = C.c_int32
+        L.memosight_last_cuda_error.restype = C.c_int32
+        L.memosight_ama.restype = C.c_int32
+        L.memosight_ama.argtypes = [C.c_int32, C.c_int32]
+        L.memosight_upl_pids.restype = C.c_int32
+        L.memosight_upl_pids.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_uint32, C.c_void_p, C.c_int32]
+        L.memosight_out_pid.restype = C.c_int32
+        L.memosight_out_pid.argtypes = [C.c_int32, C.c_int32]
+        L.memosight_step_pids.restype = C.c_int32
+        L.memosight_step_pids.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
+        L.memosight_rope_qk.restype = C.c_int32
+        L.memosight_rope_qk.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
+                                        C.c_int32, C.c_double, C.c_void_p, C.c_uint32, C.c_void_p]
+        L.memosight_attn_workspace_bytes.restype = C.c_size_t
+        L.memosight_attn_workspace_bytes.argtypes = [C.c_int32] * 6
+        L.memosight_attn_step.restype = C.c_int32
+        L.memosight_attn_step.argtypes = [C.POINTER(AttnParams), C.c_void_p]
+        L.memosight_attn_status.restype = C.c_int32
+        L.memosight_attn_status.argtypes = [C.c_void_p, C.c_void_p]
+        L.memosight_kv_compact.restype = C.c_int32
+        L.memosight_kv_compact.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int64, C.c_int64, C.c_int32,
+                                           C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
+                                           C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p]
+        L.memosight_kv_append.restype = C.c_int32
+        L.memosight_kv_append.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_int32,
+                                          C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                          C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p]
+        L.memosight_accept_workspace_bytes.restype = C.c_size_t
+        L.memosight_accept_workspace_bytes.argtypes = [C.c_int32, C.c_int32]
+        L.memosight_accept.restype = C.c_int32
+        L.memosight_accept.argtypes = [C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_int32, C.c_int32,
+                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+        _lib = L
+    return _lib
+
+
+def _ptr(t) -> Optional[int]:
+    """Address behind a tensor-like argument (marshalling only)."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    if hasattr(t, "data_ptr"):
+        if not t.is_contiguous():
+            raise ValueError("memosight: tensors must be contiguous")
+        return t.data_ptr()
+    raise TypeError(f"memosight: cannot take the address of {type(t)!r}")
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream if torch.cuda.is_available() else None
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+def _check(rc: int, what: str) -> None:
+    if rc != MS_OK:
+        raise MemosightError(rc, what)
+
+
+# ------------------------------------------------------------------ host helpers
+
+def memosight_version() -> int:
+    return int(lib().memosight_version())
+
+
+def memosight_ama(n: int, c: int) -> int:
+    r = int(lib().memosight_ama(n, c))
+    if r < 0:
+        raise MemosightError(r, "memosight_ama")
+    return r
+
+
+def memosight_upl_pids(rho_first: int, n: int, c: int, flags: int = 0) -> np.ndarray:
+    out = np.empty(max(n, 1), dtype=np.int32)
+    r = int(lib().memosight_upl_pids(rho_first, n, c, flags, out.ctypes.data, out.size))
+    if r < 0:
+        raise MemosightError(r, "memosight_upl_pids")
+    return out[:r].copy()
+
+
+def memosight_out_pid(rho_first: int, n: int) -> int:
+    return int(lib().memosight_out_pid(rho_first, n))
+
+
+def memosight_step_pids(p0: int, n_c: int, d: int, anchor: Optional[Sequence[int]] = None) -> np.ndarray:
+    out = np.empty(max(n_c + d, 1), dtype=np.int32)
+    a = None if anchor is None else np.ascontiguousarray(anchor, dtype=np.int32)
+    _check(int(lib().memosight_step_pids(p0, n_c, d, None if a is None else a.ctypes.data, out.ctypes.data)),
+           "memosight_step_pids")
+    return out[:n_c + d].copy()
+
+
+# ------------------------------------------------------------------ device calls
+
+def memosight_rope_qk(q, k, pos_id, T: int, H_q: int, H_kv: int, D: int, rope_base: float,
+                      inv_freq=None, flags: int = 0, stream=None) -> None:
+    f = None if inv_freq is None else np.ascontiguousarray(inv_freq, dtype=np.float64)
+    _check(int(lib().memosight_rope_qk(_ptr(q), _ptr(k), _ptr(pos_id), T, H_q, H_kv, D, float(rope_base),
+                                       None if f is None else f.ctypes.data, flags, _stream(stream))),
+           "memosight_rope_qk")
+
+
+def memosight_attn_workspace_bytes(batch: int, n_q_heads: int, n_kv_heads: int, head_dim: int,
+                                   max_kv_len: int, max_nq: int) -> int:
+    return int(lib().memosight_attn_workspace_bytes(batch, n_q_heads, n_kv_heads, head_dim, max_kv_len, max_nq))
+
+
+def memosight_attn_step(*, batch, n_q_heads, n_kv_heads, head_dim, k_cache, v_cache, kv_head_stride, n_slots,
+                        kv_off, kv_len, max_kv_len, max_nq, q_off, n_cand, anchor, total_rows, sm_scale,
+                        q, k_step, v_step, out, lse, workspace, workspace_bytes, stream=None) -> None:
+    p = AttnParams()
+    p.struct_size = C.sizeof(AttnParams)
+    p.batch, p.n_q_heads, p.n_kv_heads, p.head_dim = batch, n_q_heads, n_kv_heads, head_dim
+    p.k_cache, p.v_cache = _ptr(k_cache), _ptr(v_cache)
+    p.kv_head_stride, p.n_slots = kv_head_stride, n_slots
+    p.kv_off, p.kv_len = _ptr(kv_off), _ptr(kv_len)
+    p.max_kv_len, p.max_nq = max_kv_len, max_nq
+    p.q_off, p.n_cand, p.anchor = _ptr(q_off), _ptr(n_cand), _ptr(anchor)
+    p.total_rows, p.sm_scale = total_rows, float(sm_scale)
+    p.q, p.k_step, p.v_step = _ptr(q), _ptr(k_step), _ptr(v_step)
+    p.out, p.lse = _ptr(out), _ptr(lse)
+    p.workspace, p.workspace_bytes = _ptr(workspace), workspace_bytes
+    _check(int(lib().memosight_attn_step(C.byref(p), _stream(stream))), "memosight_attn_step")
+
+
+def memosight_attn_status(workspace, stream=None) -> int:
+    """Synchronises the stream; returns MS_OK or MS_ERR_DEVICE_TIMEOUT (raises on CUDA errors)."""
+    rc = int(lib().memosight_attn_status(_ptr(workspace), _stream(stream)))
+    if rc not in (MS_OK, MS_ERR_DEVICE_TIMEOUT):
+        raise MemosightError(rc, "memosight_attn_status")
+    return rc
+
+
+def memosight_kv_compact(k_cache, v_cache, n_layers, layer_stride, kv_head_stride, batch, n_kv_heads, head_dim,
+                         kv_off, kv_len, seg_start, seg_len, src_idx, idx_stride, max_tail, stream=None) -> None:
+    _check(int(lib().memosight_kv_compact(_ptr(k_cache), _ptr(v_cache), n_layers, layer_stride, kv_head_stride,
+                                          batch, n_kv_heads, head_dim, _ptr(kv_off), _ptr(kv_len),
+                                          _ptr(seg_start), _ptr(seg_len), _ptr(src_idx), idx_stride, max_tail,
+                                          _stream(stream))), "memosight_kv_compact")
+
+
+def memosight_kv_append(k_cache, v_cache, kv_head_stride, batch, n_kv_heads, head_dim, kv_off, kv_len, k_step,
+                        v_step, q_off, n_cand, n_keep, max_nq, bump_len, stream=None) -> None:
+    _check(int(lib().memosight_kv_append(_ptr(k_cache), _ptr(v_cache), kv_head_stride, batch, n_kv_heads,
+                                         head_dim, _ptr(kv_off), _ptr(kv_len), _ptr(k_step), _ptr(v_step),
+                                         _ptr(q_off), _ptr(n_cand), _ptr(n_keep), max_nq, int(bool(bump_len)),
+                                         _stream(stream))), "memosight_kv_append")
+
+
+def memosight_accept_workspace_bytes(total_rows: int, vocab: int) -> int:
+    return int(lib().memosight_accept_workspace_bytes(total_rows, vocab))
+
+
+def memosight_accept(logits, ld_v, vocab, row_off, batch, total_rows, draft, argmax_out, n_match, workspace,
+                     workspace_bytes, stream=None) -> None:
+    _check(int(lib().memosight_accept(_ptr(logits), ld_v, vocab, _ptr(row_off), batch, total_rows, _ptr(draft),
+                                      _ptr(argmax_out), _ptr(n_match), _ptr(workspace), workspace_bytes,
+                                      _stream(stream))), "memosight_accept")

@@ -1,0 +1,93 @@
+// Entry points of the step attention: argument validation, path selection,
+// workspace sizing and the device status word.
+#include <math.h>
+
+#include "attn_internal.cuh"
+
+namespace {
+
+bool fast_path_shape(int D, int G, int max_nq) {
+  return (D == 64 || D == 128) && max_nq * G <= 64;
+}
+
+}  // namespace
+
+extern "C" size_t memosight_attn_workspace_bytes(int32_t batch, int32_t n_q_heads,
+                                                 int32_t n_kv_heads, int32_t head_dim,
+                                                 int32_t max_kv_len, int32_t max_nq) {
+  if (batch < 0 || n_kv_heads < 1 || n_q_heads < 1 || n_q_heads % n_kv_heads || head_dim < 1 ||
+      max_kv_len < 0 || max_nq < 1 || max_nq > ms::kMaxNq)
+    return 0;
+  const int G = n_q_heads / n_kv_heads;
+  if (!fast_path_shape(head_dim, G, max_nq)) return ms::kWsHeaderBytes;
+  int n_ctas = ms::attn_mma_grid();
+  if (n_ctas <= 0) n_ctas = 256;   // no device visible: answer for the largest part we target
+  const int rows_pad = (max_nq * G + 15) & ~15;
+  return ms::attn_mma_workspace_bytes(head_dim, rows_pad, n_ctas);
+}
+
+extern "C" int32_t memosight_attn_step(const memosight_attn_params* p, memosight_stream_t stream) {
+  if (!p || p->struct_size != sizeof(memosight_attn_params)) return MS_ERR_INVALID_ARG;
+  if (p->batch < 0 || p->n_kv_heads < 1 || p->n_q_heads < 1 || p->head_dim < 1 ||
+      p->max_kv_len < 0 || p->total_rows < 0 || p->n_slots < 0 || p->kv_head_stride < 0)
+    return MS_ERR_INVALID_ARG;
+  if (p->n_q_heads % p->n_kv_heads) return MS_ERR_INVALID_ARG;
+  const int G = p->n_q_heads / p->n_kv_heads;
+  if (G > ms::kMaxGroup || p->max_nq < 1 || p->max_nq > ms::kMaxNq || p->batch > ms::kMaxBatch ||
+      p->head_dim % 32 || p->head_dim > 256 || p->n_slots >= (1ll << 31))
+    return MS_ERR_UNSUPPORTED_SHAPE;
+  if (p->batch == 0 || p->total_rows == 0) return MS_OK;
+  if (!p->kv_off || !p->kv_len || !p->q_off || !p->n_cand || !p->q || !p->k_step || !p->v_step ||
+      !p->out || !p->workspace)
+    return MS_ERR_INVALID_ARG;
+  if (p->max_kv_len > 0 && (!p->k_cache || !p->v_cache || p->n_slots < 1)) return MS_ERR_INVALID_ARG;
+  if (p->kv_head_stride < p->n_slots * p->head_dim) return MS_ERR_INVALID_ARG;
+  if (!(p->sm_scale >= 0.f) || isinf(p->sm_scale)) return MS_ERR_INVALID_ARG;
+  if (!ms::aligned16(p->k_cache) || !ms::aligned16(p->v_cache) || !ms::aligned16(p->q) ||
+      !ms::aligned16(p->k_step) || !ms::aligned16(p->v_step) || !ms::aligned16(p->out) ||
+      (p->kv_head_stride % 8) || (reinterpret_cast<uintptr_t>(p->workspace) & 255u))
+    return MS_ERR_ALIGNMENT;
+  const size_t need = memosight_attn_workspace_bytes(p->batch, p->n_q_heads, p->n_kv_heads,
+                                                     p->head_dim, p->max_kv_len, p->max_nq);
+  if (need == 0) return MS_ERR_INVALID_ARG;
+  if (p->workspace_bytes < need) return MS_ERR_WORKSPACE_TOO_SMALL;
+
+  ms::AttnArgs a;
+  a.B = p->batch; a.H_q = p->n_q_heads; a.H_kv = p->n_kv_heads; a.G = G; a.D = p->head_dim;
+  a.T = p->total_rows;
+  a.k_cache = static_cast<const __nv_bfloat16*>(p->k_cache);
+  a.v_cache = static_cast<const __nv_bfloat16*>(p->v_cache);
+  a.kv_head_stride = p->kv_head_stride;
+  a.n_slots = p->n_slots;
+  a.kv_off = p->kv_off; a.kv_len = p->kv_len; a.q_off = p->q_off; a.n_cand = p->n_cand;
+  a.anchor = p->anchor;
+  a.q = static_cast<const __nv_bfloat16*>(p->q);
+  a.k_step = static_cast<const __nv_bfloat16*>(p->k_step);
+  a.v_step = static_cast<const __nv_bfloat16*>(p->v_step);
+  a.out = static_cast<__nv_bfloat16*>(p->out);
+  a.lse = p->lse;
+  const double scale = p->sm_scale > 0.f ? static_cast<double>(p->sm_scale)
+                                         : 1.0 / sqrt(static_cast<double>(p->head_dim));
+  a.scale_log2 = static_cast<float>(scale * 1.4426950408889634);
+  a.max_kv_len = p->max_kv_len; a.max_nq = p->max_nq;
+  a.workspace = p->workspace;
+
+  cudaStream_t st = ms::as_stream(stream);
+  // An empty cache tensor still needs a valid address for the tile descriptors.
+  if (fast_path_shape(a.D, G, a.max_nq) && a.k_cache && a.v_cache && a.n_slots >= 1)
+    return ms::launch_attn_mma(a, st);
+  return ms::launch_attn_simt(a, st);
+}
+
+extern "C" int32_t memosight_attn_status(const void* workspace, memosight_stream_t stream) {
+  if (!workspace) return MS_ERR_INVALID_ARG;
+  MS_CUDA_TRY(cudaStreamSynchronize(ms::as_stream(stream)));
+  uint32_t word = 0;
+  MS_CUDA_TRY(cudaMemcpy(&word, workspace, sizeof word, cudaMemcpyDeviceToHost));
+  if (word == 0x4D535431u || word == 0x4D535432u) {
+    const uint32_t zero = 0;
+    MS_CUDA_TRY(cudaMemcpy(const_cast<void*>(workspace), &zero, sizeof zero, cudaMemcpyHostToDevice));
+    return MS_ERR_DEVICE_TIMEOUT;
+  }
+  return MS_OK;
+}

@@ -1,0 +1,43 @@
+// Internal interface between the attention entry point and its kernels.
+#pragma once
+
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace ms {
+
+// Validated, typed copy of memosight_attn_params as the kernels take it.
+struct AttnArgs {
+  int B, H_q, H_kv, G, D, T;
+  const __nv_bfloat16* k_cache;
+  const __nv_bfloat16* v_cache;
+  int64_t kv_head_stride;
+  int64_t n_slots;
+  const int64_t* kv_off;
+  const int32_t* kv_len;
+  const int32_t* q_off;
+  const int32_t* n_cand;
+  const int32_t* anchor;
+  const __nv_bfloat16* q;
+  const __nv_bfloat16* k_step;
+  const __nv_bfloat16* v_step;
+  __nv_bfloat16* out;
+  float* lse;
+  float scale_log2;   // softmax scale * log2(e): scores live in the exp2 domain
+  int max_kv_len, max_nq;
+  void* workspace;
+};
+
+// Workspace header (first 256 bytes): word 0 = device status (0 ok, 1 = a bounded
+// wait ran out), the rest reserved.
+constexpr size_t kWsHeaderBytes = 256;
+
+int32_t launch_attn_simt(const AttnArgs& a, cudaStream_t st);
+
+// Tensor-core split-KV path.  rows_pad = packed rows per KV head rounded up to 16.
+size_t attn_mma_workspace_bytes(int D, int rows_pad, int n_ctas);
+int32_t launch_attn_mma(const AttnArgs& a, cudaStream_t st);
+int attn_mma_grid();   // persistent CTAs the split kernel launches on this device
+
+}  // namespace ms

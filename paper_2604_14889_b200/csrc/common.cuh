@@ -1,0 +1,46 @@
+// Shared host/device helpers of the MemoSight CUDA library (sm_100a only).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "memosight.h"
+
+namespace ms {
+
+// Thread-local record of the last CUDA error behind an MS_ERR_CUDA.
+void set_last_cuda_error(cudaError_t e);
+
+inline int32_t cuda_status(cudaError_t e) {
+  if (e == cudaSuccess) return MS_OK;
+  set_last_cuda_error(e);
+  return MS_ERR_CUDA;
+}
+
+#define MS_CUDA_TRY(expr)                              \
+  do {                                                 \
+    cudaError_t e__ = (expr);                          \
+    if (e__ != cudaSuccess) return ms::cuda_status(e__); \
+  } while (0)
+
+// Launch check: launch-configuration errors surface through cudaGetLastError.
+#define MS_LAUNCH_CHECK() MS_CUDA_TRY(cudaGetLastError())
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Number of SMs of the current device (cached per device).
+int32_t sm_count();
+
+inline cudaStream_t as_stream(memosight_stream_t s) { return reinterpret_cast<cudaStream_t>(s); }
+
+constexpr int kMaxNq = 16;        // largest step block
+constexpr int kMaxGroup = 16;     // largest H_q / H_kv
+constexpr int kMaxBatch = 8192;   // sequences per attention launch
+
+// Step-local visibility (see memosight_attn_params): key j of the block vs row i.
+__host__ __device__ inline bool step_key_visible(int i, int j, int n_c, int a_i) {
+  return (j == i) || (j < n_c && j < a_i);
+}
+
+}  // namespace ms

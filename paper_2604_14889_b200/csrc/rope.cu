@@ -1,0 +1,102 @@
+// RoPE applied in place to the step block's Q and K at token-specific position
+// IDs (paper Sec. 2.1.2: the position layouts of memory and foresight tokens act
+// through RoPE, so each new token is rotated by its own PID, not by its cache slot).
+//
+// One CTA per token.  The D/2 angles of the token are evaluated once in fp64
+// (sincos of pos * theta_i), kept in shared memory and reused by all H_q + H_kv
+// heads; the rotation is done in fp64 and rounded to bf16 once, so the result
+// equals an fp64 reference up to the last-bit behaviour of sin/cos.
+#include <math.h>
+
+#include "common.cuh"
+
+namespace {
+
+constexpr int kMaxHalf = 128;  // D <= 256
+
+struct FreqTable {
+  double f[kMaxHalf];
+};
+
+__device__ __forceinline__ uint16_t f64_to_bf16_bits(double x) {
+  // One rounding fp64 -> bf16 (round to nearest even).  Going through fp32
+  // would round twice; instead round the fp64 significand directly: bf16 keeps
+  // 8 significant bits, i.e. drops the low 45 bits of the 53-bit significand.
+  if (x != x) return 0x7FC0;
+  const double ax = fabs(x);
+  if (ax >= 3.3961775292304601e38) {            // >= max bf16 + half ulp: overflow to inf
+    return static_cast<uint16_t>((x < 0 ? 0x8000u : 0u) | 0x7F80u);
+  }
+  if (ax < 1.1754943508222875e-38) {            // below the smallest normal: fixed spacing 2^-133
+    const double q = rint(ax * 0x1p133);         // exact scaling, RNE
+    const uint32_t m = static_cast<uint32_t>(q); // 0 .. 128 (128 = smallest normal)
+    return static_cast<uint16_t>((x < 0 ? 0x8000u : 0u) | m);
+  }
+  uint64_t b = static_cast<uint64_t>(__double_as_longlong(ax));
+  const uint64_t drop = 45;
+  const uint64_t half = 1ull << (drop - 1);
+  const uint64_t rem = b & ((1ull << drop) - 1);
+  b >>= drop;                                     // exponent(11) | top 7 mantissa bits
+  if (rem > half || (rem == half && (b & 1))) b += 1;   // carries into the exponent correctly
+  const int32_t e = static_cast<int32_t>(b >> 7) - 1023 + 127;   // rebias
+  const uint32_t out = (static_cast<uint32_t>(e) << 7) | static_cast<uint32_t>(b & 0x7F);
+  return static_cast<uint16_t>((x < 0 ? 0x8000u : 0u) | out);
+}
+
+__device__ __forceinline__ double bf16_bits_to_f64(uint16_t h) {
+  return static_cast<double>(__uint_as_float(static_cast<uint32_t>(h) << 16));
+}
+
+__global__ void __launch_bounds__(128)
+rope_qk_kernel(uint16_t* __restrict__ q, uint16_t* __restrict__ k, const int32_t* __restrict__ pos_id,
+               int H_q, int H_kv, int D, uint32_t flags, FreqTable freq) {
+  __shared__ double s_cos[kMaxHalf];
+  __shared__ double s_sin[kMaxHalf];
+  const int t = blockIdx.x;
+  const int half = D >> 1;
+  double p = static_cast<double>(pos_id[t]);
+  if (flags & MS_POS_HALF_UNITS) p *= 0.5;
+  for (int i = threadIdx.x; i < half; i += blockDim.x) {
+    double s, c;
+    sincos(p * freq.f[i], &s, &c);
+    s_cos[i] = c;
+    s_sin[i] = s;
+  }
+  __syncthreads();
+  const bool interleaved = (flags & MS_ROPE_INTERLEAVED) != 0;
+  const int n_heads = H_q + H_kv;
+  for (int w = threadIdx.x; w < n_heads * half; w += blockDim.x) {
+    const int h = w / half, i = w - h * half;
+    uint16_t* v = (h < H_q) ? q + (static_cast<int64_t>(t) * H_q + h) * D
+                            : k + (static_cast<int64_t>(t) * H_kv + (h - H_q)) * D;
+    const int ia = interleaved ? 2 * i : i;
+    const int ib = interleaved ? 2 * i + 1 : i + half;
+    const double a = bf16_bits_to_f64(v[ia]), b = bf16_bits_to_f64(v[ib]);
+    const double c = s_cos[i], s = s_sin[i];
+    v[ia] = f64_to_bf16_bits(a * c - b * s);
+    v[ib] = f64_to_bf16_bits(b * c + a * s);
+  }
+}
+
+}  // namespace
+
+extern "C" int32_t memosight_rope_qk(void* q, void* k, const int32_t* pos_id, int32_t T, int32_t H_q,
+                                     int32_t H_kv, int32_t D, double rope_base,
+                                     const double* inv_freq, uint32_t flags,
+                                     memosight_stream_t stream) {
+  if (T < 0 || H_q < 0 || H_kv < 0) return MS_ERR_INVALID_ARG;
+  if (D < 2 || (D & 1) || D > 2 * kMaxHalf) return MS_ERR_UNSUPPORTED_SHAPE;
+  if (flags & ~(MS_ROPE_INTERLEAVED | MS_POS_HALF_UNITS)) return MS_ERR_INVALID_ARG;
+  if (T == 0 || H_q + H_kv == 0) return MS_OK;
+  if (!pos_id || (H_q > 0 && !q) || (H_kv > 0 && !k)) return MS_ERR_INVALID_ARG;
+  if (!inv_freq && !(rope_base > 0.0)) return MS_ERR_INVALID_ARG;
+  FreqTable freq;
+  for (int i = 0; i < D / 2; ++i)
+    freq.f[i] = inv_freq ? inv_freq[i] : pow(rope_base, -2.0 * static_cast<double>(i) / D);
+  for (int i = D / 2; i < kMaxHalf; ++i) freq.f[i] = 0.0;
+  rope_qk_kernel<<<T, 128, 0, ms::as_stream(stream)>>>(static_cast<uint16_t*>(q),
+                                                        static_cast<uint16_t*>(k), pos_id, H_q, H_kv,
+                                                        D, flags, freq);
+  MS_LAUNCH_CHECK();
+  return MS_OK;
+}
