@@ -144,6 +144,8 @@ typedef struct memosight_attn_params {
   float* lse;                /* device fp32 [T][H_q], natural-log sum-exp, or NULL             */
   void* workspace;           /* device scratch, 256-byte aligned                               */
   size_t workspace_bytes;    /* >= memosight_attn_workspace_bytes(...)                         */
+  void* ev_split_begin;      /* optional cudaEvent_t recorded on `stream` right before ...     */
+  void* ev_split_end;        /* ... and right after the split-KV kernel (NULL: not recorded)   */
 } memosight_attn_params;
 
 /* Scratch size for memosight_attn_step with these bounds (0 on invalid input).
@@ -213,13 +215,58 @@ MS_API size_t memosight_accept_workspace_bytes(int32_t total_rows, int32_t vocab
  *              larger than any number and the first NaN wins
  *   n_match    device int32 [B]: largest m with draft >= 0 and argmax == draft on
  *              the block's rows 0..m-1
+ *   n_keep     device int32 [B] or NULL: n_match + 1 (0 for an empty block), the
+ *              number of candidates that become permanent -- what kv_append takes
  * Row convention: row i of a block holds candidate c_i and predicts the token
  * after it, so draft[i] = c_{i+1}; tokens c_0..c_{n_match} become permanent and
  * argmax_out[row n_match] is the next token. */
 MS_API int32_t memosight_accept(const float* logits, int64_t ld_v, int32_t vocab, const int32_t* row_off,
                          int32_t batch, int32_t total_rows, const int32_t* draft,
-                         int32_t* argmax_out, int32_t* n_match, void* workspace,
+                         int32_t* argmax_out, int32_t* n_match, int32_t* n_keep, void* workspace,
                          size_t workspace_bytes, memosight_stream_t stream);
+
+/* ---- One whole step with the step's inputs and results in host memory -------------------- */
+
+/* The KV cache is device-resident state (it is what the method keeps compacted);
+ * everything a step consumes or produces besides it may live on the host.  This
+ * call copies the step's inputs from host memory (pinned memory makes the copies
+ * asynchronous), runs RoPE -> step attention -> greedy accept -> append of the
+ * accepted candidates (-> optional compaction) on `stream`, and copies the results
+ * back.  All device pointers are caller-owned staging buffers of the stated sizes.
+ * The call returns after queueing; synchronise `stream` before reading h_*. */
+typedef struct memosight_step_host_params {
+  uint32_t struct_size;          /* sizeof(memosight_step_host_params)                         */
+  memosight_attn_params attn;    /* device-side description of the step: q, k_step, v_step, out,
+                                    lse are the device staging buffers the host data goes
+                                    through; k_cache/v_cache/kv_len are updated by the append  */
+  const void* h_q;               /* host bf16 [T][H_q][D], before RoPE                         */
+  const void* h_k_step;          /* host bf16 [T][H_kv][D], before RoPE                        */
+  const void* h_v_step;          /* host bf16 [T][H_kv][D]                                     */
+  const int32_t* h_pos_id;       /* host [T] position IDs of the block rows                    */
+  int32_t* d_pos_id;             /* device [T] staging                                         */
+  double rope_base;              /* theta_i = rope_base^(-2i/D)                                */
+  uint32_t rope_flags;           /* MS_ROPE_* | MS_POS_*                                       */
+  int32_t vocab;                 /* V; 0 skips accept and append                               */
+  const float* h_logits;         /* host fp32 [T][ld_v]                                        */
+  int64_t ld_v;
+  float* d_logits;               /* device [T][ld_v] staging                                   */
+  const int32_t* h_draft;        /* host [T]                                                   */
+  int32_t* d_draft;              /* device [T] staging                                         */
+  int32_t* d_argmax;             /* device [T]                                                 */
+  int32_t* d_n_match;            /* device [B]                                                 */
+  int32_t* d_n_keep;             /* device [B]                                                 */
+  void* accept_workspace;        /* device, memosight_accept_workspace_bytes(T, V)             */
+  size_t accept_workspace_bytes;
+  const int32_t* d_seg_start;    /* device [B] or NULL: compaction request after the append    */
+  const int32_t* d_seg_len;      /* device [B] (0 = skip sequence) when d_seg_start != NULL    */
+  int32_t max_tail;              /* host bound of the entries a compaction moves               */
+  void* h_out;                   /* host bf16 [T][H_q][D]                                      */
+  int32_t* h_argmax;             /* host [T] or NULL                                           */
+  int32_t* h_n_match;            /* host [B] or NULL                                           */
+} memosight_step_host_params;
+
+MS_API int32_t memosight_step_host(const memosight_step_host_params* params,
+                                   memosight_stream_t stream);
 
 #ifdef __cplusplus
 }

@@ -55,6 +55,23 @@ class AttnParams(C.Structure):
         ("q", C.c_void_p), ("k_step", C.c_void_p), ("v_step", C.c_void_p),
         ("out", C.c_void_p), ("lse", C.c_void_p),
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+        ("ev_split_begin", C.c_void_p), ("ev_split_end", C.c_void_p),
+    ]
+
+
+class StepHostParams(C.Structure):
+    """Mirror of ``memosight_step_host_params`` (include/memosight.h)."""
+    _fields_ = [
+        ("struct_size", C.c_uint32), ("attn", AttnParams),
+        ("h_q", C.c_void_p), ("h_k_step", C.c_void_p), ("h_v_step", C.c_void_p),
+        ("h_pos_id", C.c_void_p), ("d_pos_id", C.c_void_p),
+        ("rope_base", C.c_double), ("rope_flags", C.c_uint32), ("vocab", C.c_int32),
+        ("h_logits", C.c_void_p), ("ld_v", C.c_int64), ("d_logits", C.c_void_p),
+        ("h_draft", C.c_void_p), ("d_draft", C.c_void_p),
+        ("d_argmax", C.c_void_p), ("d_n_match", C.c_void_p), ("d_n_keep", C.c_void_p),
+        ("accept_workspace", C.c_void_p), ("accept_workspace_bytes", C.c_size_t),
+        ("d_seg_start", C.c_void_p), ("d_seg_len", C.c_void_p), ("max_tail", C.c_int32),
+        ("h_out", C.c_void_p), ("h_argmax", C.c_void_p), ("h_n_match", C.c_void_p),
     ]
 
 
@@ -102,7 +119,10 @@ def lib() -> C.CDLL:
         L.memosight_accept_workspace_bytes.argtypes = [C.c_int32, C.c_int32]
         L.memosight_accept.restype = C.c_int32
         L.memosight_accept.argtypes = [C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_int32, C.c_int32,
-                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
+                                       C.c_void_p]
+        L.memosight_step_host.restype = C.c_int32
+        L.memosight_step_host.argtypes = [C.POINTER(StepHostParams), C.c_void_p]
         _lib = L
     return _lib
 
@@ -182,9 +202,11 @@ def memosight_attn_workspace_bytes(batch: int, n_q_heads: int, n_kv_heads: int, 
     return int(lib().memosight_attn_workspace_bytes(batch, n_q_heads, n_kv_heads, head_dim, max_kv_len, max_nq))
 
 
-def memosight_attn_step(*, batch, n_q_heads, n_kv_heads, head_dim, k_cache, v_cache, kv_head_stride, n_slots,
-                        kv_off, kv_len, max_kv_len, max_nq, q_off, n_cand, anchor, total_rows, sm_scale,
-                        q, k_step, v_step, out, lse, workspace, workspace_bytes, stream=None) -> None:
+def attn_params(*, batch, n_q_heads, n_kv_heads, head_dim, k_cache, v_cache, kv_head_stride, n_slots,
+                kv_off, kv_len, max_kv_len, max_nq, q_off, n_cand, anchor, total_rows, sm_scale,
+                q, k_step, v_step, out, lse, workspace, workspace_bytes, ev_split_begin=None,
+                ev_split_end=None) -> AttnParams:
+    """Fills a memosight_attn_params structure (addresses only; nothing is copied)."""
     p = AttnParams()
     p.struct_size = C.sizeof(AttnParams)
     p.batch, p.n_q_heads, p.n_kv_heads, p.head_dim = batch, n_q_heads, n_kv_heads, head_dim
@@ -197,7 +219,18 @@ def memosight_attn_step(*, batch, n_q_heads, n_kv_heads, head_dim, k_cache, v_ca
     p.q, p.k_step, p.v_step = _ptr(q), _ptr(k_step), _ptr(v_step)
     p.out, p.lse = _ptr(out), _ptr(lse)
     p.workspace, p.workspace_bytes = _ptr(workspace), workspace_bytes
+    p.ev_split_begin, p.ev_split_end = _ptr(ev_split_begin), _ptr(ev_split_end)
+    return p
+
+
+def memosight_attn_step(params: Optional[AttnParams] = None, stream=None, **fields) -> None:
+    """memosight_attn_step(params) or memosight_attn_step(**fields of attn_params)."""
+    p = params if params is not None else attn_params(**fields)
     _check(int(lib().memosight_attn_step(C.byref(p), _stream(stream))), "memosight_attn_step")
+
+
+def memosight_step_host(params: StepHostParams, stream=None) -> None:
+    _check(int(lib().memosight_step_host(C.byref(params), _stream(stream))), "memosight_step_host")
 
 
 def memosight_attn_status(workspace, stream=None) -> int:
@@ -228,8 +261,8 @@ def memosight_accept_workspace_bytes(total_rows: int, vocab: int) -> int:
     return int(lib().memosight_accept_workspace_bytes(total_rows, vocab))
 
 
-def memosight_accept(logits, ld_v, vocab, row_off, batch, total_rows, draft, argmax_out, n_match, workspace,
-                     workspace_bytes, stream=None) -> None:
+def memosight_accept(logits, ld_v, vocab, row_off, batch, total_rows, draft, argmax_out, n_match, n_keep,
+                     workspace, workspace_bytes, stream=None) -> None:
     _check(int(lib().memosight_accept(_ptr(logits), ld_v, vocab, _ptr(row_off), batch, total_rows, _ptr(draft),
-                                      _ptr(argmax_out), _ptr(n_match), _ptr(workspace), workspace_bytes,
-                                      _stream(stream))), "memosight_accept")
+                                      _ptr(argmax_out), _ptr(n_match), _ptr(n_keep), _ptr(workspace),
+                                      workspace_bytes, _stream(stream))), "memosight_accept")

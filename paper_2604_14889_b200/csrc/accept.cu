@@ -95,7 +95,7 @@ argmax_chunks_kernel(const float* __restrict__ logits, int64_t ld_v, int V, int 
 __global__ void __launch_bounds__(128)
 accept_rows_kernel(const Cand* __restrict__ part, int n_chunks, const int32_t* __restrict__ row_off,
                    int B, const int32_t* __restrict__ draft, int32_t* __restrict__ argmax_out,
-                   int32_t* __restrict__ n_match) {
+                   int32_t* __restrict__ n_match, int32_t* __restrict__ n_keep) {
   const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (b >= B) return;
@@ -117,6 +117,7 @@ accept_rows_kernel(const Cand* __restrict__ part, int n_chunks, const int32_t* _
       ++m;
     }
     n_match[b] = m;
+    if (n_keep) n_keep[b] = (r1 > r0) ? m + 1 : 0;   // c_0 .. c_m become permanent
   }
 }
 
@@ -133,7 +134,7 @@ extern "C" size_t memosight_accept_workspace_bytes(int32_t total_rows, int32_t v
 extern "C" int32_t memosight_accept(const float* logits, int64_t ld_v, int32_t vocab,
                                     const int32_t* row_off, int32_t batch, int32_t total_rows,
                                     const int32_t* draft, int32_t* argmax_out, int32_t* n_match,
-                                    void* workspace, size_t workspace_bytes,
+                                    int32_t* n_keep, void* workspace, size_t workspace_bytes,
                                     memosight_stream_t stream) {
   if (batch < 0 || total_rows < 0 || vocab < 1 || ld_v < vocab) return MS_ERR_INVALID_ARG;
   if (batch == 0) return total_rows == 0 ? MS_OK : MS_ERR_INVALID_ARG;
@@ -157,7 +158,7 @@ extern "C" int32_t memosight_accept(const float* logits, int64_t ld_v, int32_t v
     MS_LAUNCH_CHECK();
   }
   accept_rows_kernel<<<(batch + 3) / 4, 128, 0, st>>>(part, n_chunks, row_off, batch, draft,
-                                                      argmax_out, n_match);
+                                                      argmax_out, n_match, n_keep);
   MS_LAUNCH_CHECK();
   return MS_OK;
 }

@@ -71,6 +71,8 @@ extern "C" int32_t memosight_attn_step(const memosight_attn_params* p, memosight
   a.scale_log2 = static_cast<float>(scale * 1.4426950408889634);
   a.max_kv_len = p->max_kv_len; a.max_nq = p->max_nq;
   a.workspace = p->workspace;
+  a.ev_split_begin = static_cast<cudaEvent_t>(p->ev_split_begin);
+  a.ev_split_end = static_cast<cudaEvent_t>(p->ev_split_end);
 
   cudaStream_t st = ms::as_stream(stream);
   // An empty cache tensor still needs a valid address for the tile descriptors.

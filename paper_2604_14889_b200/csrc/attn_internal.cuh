@@ -27,6 +27,7 @@ struct AttnArgs {
   float scale_log2;   // softmax scale * log2(e): scores live in the exp2 domain
   int max_kv_len, max_nq;
   void* workspace;
+  cudaEvent_t ev_split_begin, ev_split_end;   // optional timing events around the split kernel
 };
 
 // Workspace header (first 256 bytes): word 0 = device status (0 ok, 1 = a bounded

@@ -699,8 +699,10 @@ int32_t launch_split(const AttnArgs& a, cudaStream_t st, int rows_pad, int grid,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
     configured[dev] = true;
   }
+  if (a.ev_split_begin) MS_CUDA_TRY(cudaEventRecord(a.ev_split_begin, st));
   attn_split_kernel<D, MB><<<grid, kThreads, C::SMEM_BYTES, st>>>(a, mk, mv, mks, mvs, rows_pad);
   MS_LAUNCH_CHECK();
+  if (a.ev_split_end) MS_CUDA_TRY(cudaEventRecord(a.ev_split_end, st));
   return MS_OK;
 }
 

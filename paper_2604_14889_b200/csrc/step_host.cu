@@ -1,0 +1,70 @@
+// One whole decode step driven from host-resident step data: copies in, the
+// kernels of the hot path in their order (Algorithm 1: forward pass attention,
+// greedy accept, S <- S (+) A, optional UpdateCache), copies out.  Pure
+// sequencing of the other entry points on one stream.
+#include "common.cuh"
+
+extern "C" int32_t memosight_step_host(const memosight_step_host_params* p,
+                                       memosight_stream_t stream) {
+  if (!p || p->struct_size != sizeof(memosight_step_host_params)) return MS_ERR_INVALID_ARG;
+  const memosight_attn_params& a = p->attn;
+  if (a.struct_size != sizeof(memosight_attn_params)) return MS_ERR_INVALID_ARG;
+  const int32_t T = a.total_rows, B = a.batch;
+  if (T < 0 || B < 0 || a.n_q_heads < 1 || a.n_kv_heads < 1 || a.head_dim < 1 || p->vocab < 0)
+    return MS_ERR_INVALID_ARG;
+  if (T == 0 || B == 0) return MS_OK;
+  if (!p->h_q || !p->h_k_step || !p->h_v_step || !p->h_pos_id || !p->d_pos_id || !p->h_out || !a.q ||
+      !a.k_step || !a.v_step || !a.out)
+    return MS_ERR_INVALID_ARG;
+  if (p->vocab > 0 && (!p->h_logits || !p->d_logits || !p->h_draft || !p->d_draft || !p->d_argmax ||
+                       !p->d_n_match || !p->d_n_keep || p->ld_v < p->vocab))
+    return MS_ERR_INVALID_ARG;
+  cudaStream_t st = ms::as_stream(stream);
+  const size_t q_bytes = static_cast<size_t>(T) * a.n_q_heads * a.head_dim * 2;
+  const size_t kv_bytes = static_cast<size_t>(T) * a.n_kv_heads * a.head_dim * 2;
+  // ---- host -> device: the step's inputs
+  MS_CUDA_TRY(cudaMemcpyAsync(const_cast<void*>(a.q), p->h_q, q_bytes, cudaMemcpyHostToDevice, st));
+  MS_CUDA_TRY(cudaMemcpyAsync(const_cast<void*>(a.k_step), p->h_k_step, kv_bytes, cudaMemcpyHostToDevice, st));
+  MS_CUDA_TRY(cudaMemcpyAsync(const_cast<void*>(a.v_step), p->h_v_step, kv_bytes, cudaMemcpyHostToDevice, st));
+  MS_CUDA_TRY(cudaMemcpyAsync(p->d_pos_id, p->h_pos_id, sizeof(int32_t) * T, cudaMemcpyHostToDevice, st));
+  if (p->vocab > 0) {
+    MS_CUDA_TRY(cudaMemcpyAsync(p->d_logits, p->h_logits, sizeof(float) * static_cast<size_t>(T) * p->ld_v,
+                                cudaMemcpyHostToDevice, st));
+    MS_CUDA_TRY(cudaMemcpyAsync(p->d_draft, p->h_draft, sizeof(int32_t) * T, cudaMemcpyHostToDevice, st));
+  }
+  // ---- the hot path
+  int32_t rc = memosight_rope_qk(const_cast<void*>(a.q), const_cast<void*>(a.k_step), p->d_pos_id, T,
+                                 a.n_q_heads, a.n_kv_heads, a.head_dim, p->rope_base, nullptr,
+                                 p->rope_flags, stream);
+  if (rc != MS_OK) return rc;
+  rc = memosight_attn_step(&a, stream);
+  if (rc != MS_OK) return rc;
+  if (p->vocab > 0) {
+    rc = memosight_accept(p->d_logits, p->ld_v, p->vocab, a.q_off, B, T, p->d_draft, p->d_argmax,
+                          p->d_n_match, p->d_n_keep, p->accept_workspace, p->accept_workspace_bytes,
+                          stream);
+    if (rc != MS_OK) return rc;
+    rc = memosight_kv_append(const_cast<void*>(a.k_cache), const_cast<void*>(a.v_cache),
+                             a.kv_head_stride, B, a.n_kv_heads, a.head_dim, a.kv_off,
+                             const_cast<int32_t*>(a.kv_len), a.k_step, a.v_step, a.q_off, a.n_cand,
+                             p->d_n_keep, a.max_nq, 1, stream);
+    if (rc != MS_OK) return rc;
+  }
+  if (p->d_seg_start) {
+    if (!p->d_seg_len) return MS_ERR_INVALID_ARG;
+    rc = memosight_kv_compact(const_cast<void*>(a.k_cache), const_cast<void*>(a.v_cache), 1, 0,
+                              a.kv_head_stride, B, a.n_kv_heads, a.head_dim, a.kv_off,
+                              const_cast<int32_t*>(a.kv_len), p->d_seg_start, p->d_seg_len, nullptr, 0,
+                              p->max_tail, stream);
+    if (rc != MS_OK) return rc;
+  }
+  // ---- device -> host: the step's results
+  MS_CUDA_TRY(cudaMemcpyAsync(p->h_out, a.out, q_bytes, cudaMemcpyDeviceToHost, st));
+  if (p->vocab > 0) {
+    if (p->h_argmax)
+      MS_CUDA_TRY(cudaMemcpyAsync(p->h_argmax, p->d_argmax, sizeof(int32_t) * T, cudaMemcpyDeviceToHost, st));
+    if (p->h_n_match)
+      MS_CUDA_TRY(cudaMemcpyAsync(p->h_n_match, p->d_n_match, sizeof(int32_t) * B, cudaMemcpyDeviceToHost, st));
+  }
+  return MS_OK;
+}

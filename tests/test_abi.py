@@ -45,7 +45,7 @@ def test_host_side_validation_codes():
     assert L.memosight_rope_qk(None, None, None, 4, 1, 1, 63, 1e4, None, 0, None) == ms.MS_ERR_UNSUPPORTED_SHAPE
     assert L.memosight_rope_qk(None, None, None, 4, 1, 1, 64, 1e4, None, 0, None) == ms.MS_ERR_INVALID_ARG
     assert L.memosight_rope_qk(None, None, None, 0, 1, 1, 64, 1e4, None, 0, None) == ms.MS_OK
-    assert L.memosight_accept(None, 10, 20, None, 1, 1, None, None, None, None, 0, None) == ms.MS_ERR_INVALID_ARG
+    assert L.memosight_accept(None, 10, 20, None, 1, 1, None, None, None, None, None, 0, None) == ms.MS_ERR_INVALID_ARG
     assert L.memosight_accept_workspace_bytes(-1, 5) == 0
     assert L.memosight_accept_workspace_bytes(6, 1024) >= 6 * 8
     assert L.memosight_kv_compact(None, None, 1, 0, 0, 1, 1, 12, None, None, None, None, None, 0, 0, None) \

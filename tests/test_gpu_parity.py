@@ -218,13 +218,16 @@ def _accept_both(logits, V, row_off, draft):
     want_am, want_nm = oracle.accept(logits.cpu().numpy(), V, row_off, draft)
     g_am = torch.full((T + 1,), -7, dtype=torch.int32, device=DEV)
     g_nm = torch.full((B + 1,), -7, dtype=torch.int32, device=DEV)
+    g_nk = torch.full((B,), -7, dtype=torch.int32, device=DEV)
     wsb = ms.memosight_accept_workspace_bytes(T, V)
     ws = torch.empty(wsb, dtype=torch.uint8, device=DEV)
     ms.memosight_accept(logits.to(DEV), ld, V, torch.tensor(row_off, dtype=torch.int32, device=DEV), B, T,
-                        torch.tensor(draft, dtype=torch.int32, device=DEV), g_am, g_nm, ws, wsb)
+                        torch.tensor(draft, dtype=torch.int32, device=DEV), g_am, g_nm, g_nk, ws, wsb)
     torch.cuda.synchronize()
     assert np.array_equal(g_am[:T].cpu().numpy(), want_am)
     assert np.array_equal(g_nm[:B].cpu().numpy(), want_nm)
+    rows = np.diff(np.asarray(row_off))
+    assert np.array_equal(g_nk.cpu().numpy(), np.where(rows > 0, want_nm + 1, 0))
     assert int(g_am[T]) == -7 and int(g_nm[B]) == -7
     return want_am, want_nm
 
@@ -294,13 +297,14 @@ def test_whole_step_chain_rope_attn_accept_append():
     T = B * nq
     am = torch.empty(T, dtype=torch.int32, device=DEV)
     nm = torch.empty(B, dtype=torch.int32, device=DEV)
+    nk = torch.empty(B, dtype=torch.int32, device=DEV)
     wsb = ms.memosight_accept_workspace_bytes(T, cfg.vocab)
     ws = torch.empty(wsb, dtype=torch.uint8, device=DEV)
     ms.memosight_accept(acc.logits.to(DEV), acc.ld_v, cfg.vocab, acc.row_off.to(DEV), B, T, acc.draft.to(DEV),
-                        am, nm, ws, wsb)
+                        am, nm, nk, ws, wsb)
     gk, gv, g_len = inp.k_cache[0].to(DEV).clone(), inp.v_cache[0].to(DEV).clone(), inp.kv_len.to(DEV).clone()
     ms.memosight_kv_append(gk, gv, inp.n_slots * 128, B, 2, 128, inp.kv_off.to(DEV), g_len, ks, vs,
-                           inp.q_off.to(DEV), inp.n_cand.to(DEV), nm + 1, nq, 1)
+                           inp.q_off.to(DEV), inp.n_cand.to(DEV), nk, nq, 1)
     torch.cuda.synchronize()
     assert np.array_equal(am.cpu().numpy(), am_o) and np.array_equal(nm.cpu().numpy(), nm_o)
     assert np.array_equal(g_len.cpu().numpy(), len_o)
