@@ -259,6 +259,20 @@ def workload_config(cfg, args):
             "parallelism": f"dp{args.gpus} (independent replicas by sequence, no collective on the data path)"}
 
 
+# --------------------------------------------------------------------------- multi-rank aggregation
+
+def whole_job_throughput(units_per_rank: int, elapsed_ms_local: float, world: int, device="cpu") -> tuple:
+    """Weak-scaling aggregate: every rank processed `units_per_rank` units; the job's
+    time is the slowest rank's.  Returns (units/s over all ranks, max elapsed ms)."""
+    elapsed = float(elapsed_ms_local)
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([elapsed], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed = float(t.item())
+    return world * units_per_rank / (elapsed * 1e-3), elapsed
+
+
 # --------------------------------------------------------------------------- our arm
 
 def main():
@@ -363,12 +377,7 @@ def main():
     assert inp.kv_len.cpu().tolist() == lens_after, "cache lengths differ from the replayed schedule"
     assert nm.cpu().tolist() == [k - 1 for k in sched.keep]
 
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
-    value = world * T * K / (elapsed_ms * 1e-3)
+    value, elapsed_ms = whole_job_throughput(T * K, elapsed_ms, world, dev)
 
     # roofline of the dominant kernel (split-KV attention): algorithmic KV bytes per launch / its duration
     kv_bytes = [sched.kv_bytes(W + s, cfg) for s in range(K)]

@@ -30,8 +30,8 @@ struct AttnArgs {
   cudaEvent_t ev_split_begin, ev_split_end;   // optional timing events around the split kernel
 };
 
-// Workspace header (first 256 bytes): word 0 = device status (0 ok, 1 = a bounded
-// wait ran out), the rest reserved.
+// Workspace header (first 256 bytes): word 0 = device status -- a magic value when a
+// bounded wait ran out, anything else means ok (the workspace need not be cleared).
 constexpr size_t kWsHeaderBytes = 256;
 
 int32_t launch_attn_simt(const AttnArgs& a, cudaStream_t st);
