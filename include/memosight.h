@@ -225,6 +225,35 @@ MS_API int32_t memosight_accept(const float* logits, int64_t ld_v, int32_t vocab
                          int32_t* argmax_out, int32_t* n_match, int32_t* n_keep, void* workspace,
                          size_t workspace_bytes, memosight_stream_t stream);
 
+/* Same result as memosight_accept, for callers that cannot allocate.  (The paper has no
+ * counterpart to this call; it exists for deployment reasons only.)
+ *
+ * Who needs it: a serving loop whose device memory was carved up at start-up and whose allocator
+ * is frozen while requests are in flight, a plug-in that receives tensors but no allocator, or
+ * any place where a cudaMalloc would stall the device in the middle of a decode step.  Such a
+ * caller has no workspace to hand over, so the per-chunk candidates of the argmax live in a fixed
+ * 512 KB array that is part of the library image: every GPU that loads the library holds it until
+ * the process exits.  The call itself allocates nothing -- no cudaMalloc/cudaFree, no allocating
+ * library routine -- and takes the same inputs and outputs as memosight_accept, minus the
+ * workspace.
+ *
+ * Limit: total_rows * ceil(vocab / 8192) <= MS_ACCEPT_STATIC_MAX_PARTIALS, e.g. 3449 rows at a
+ * vocabulary of 151 936.  Larger problems return MS_ERR_UNSUPPORTED_SHAPE and launch nothing;
+ * use memosight_accept with a caller workspace for those.
+ *
+ * First call on a device: the array's device address is looked up (cudaGetSymbolAddress, with
+ * that device current) and remembered; make this first call outside any stream capture.
+ *
+ * Sharing: all calls on a device use the one array, which keeps whatever the previous call left.
+ * That is harmless for sequential calls (every entry that is read is written first by the same
+ * call; nothing relies on zeros), but two calls whose kernels overlap on the GPU -- different
+ * streams, or graphs replayed concurrently -- race on it and both results are then undefined. */
+#define MS_ACCEPT_STATIC_MAX_PARTIALS 65536
+MS_API int32_t memosight_accept_static(const float* logits, int64_t ld_v, int32_t vocab,
+                                       const int32_t* row_off, int32_t batch, int32_t total_rows,
+                                       const int32_t* draft, int32_t* argmax_out, int32_t* n_match,
+                                       int32_t* n_keep, memosight_stream_t stream);
+
 /* ---- One whole step with the step's inputs and results in host memory -------------------- */
 
 /* The KV cache is device-resident state (it is what the method keeps compacted);

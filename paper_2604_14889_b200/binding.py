@@ -121,6 +121,9 @@ def lib() -> C.CDLL:
         L.memosight_accept.argtypes = [C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_int32, C.c_int32,
                                        C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
                                        C.c_void_p]
+        L.memosight_accept_static.restype = C.c_int32
+        L.memosight_accept_static.argtypes = [C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_int32, C.c_int32,
+                                              C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.memosight_step_host.restype = C.c_int32
         L.memosight_step_host.argtypes = [C.POINTER(StepHostParams), C.c_void_p]
         _lib = L
@@ -266,3 +269,16 @@ def memosight_accept(logits, ld_v, vocab, row_off, batch, total_rows, draft, arg
     _check(int(lib().memosight_accept(_ptr(logits), ld_v, vocab, _ptr(row_off), batch, total_rows, _ptr(draft),
                                       _ptr(argmax_out), _ptr(n_match), _ptr(n_keep), _ptr(workspace),
                                       workspace_bytes, _stream(stream))), "memosight_accept")
+
+
+MS_ACCEPT_STATIC_MAX_PARTIALS = 65536
+
+
+def memosight_accept_static(logits, ld_v, vocab, row_off, batch, total_rows, draft, argmax_out, n_match, n_keep,
+                            stream=None) -> None:
+    """memosight_accept for callers that cannot allocate: no workspace argument, the
+    scratch is a fixed array inside the library (see include/memosight.h for the limit,
+    the first-call rule and why concurrent calls on one GPU must not overlap)."""
+    _check(int(lib().memosight_accept_static(_ptr(logits), ld_v, vocab, _ptr(row_off), batch, total_rows,
+                                             _ptr(draft), _ptr(argmax_out), _ptr(n_match), _ptr(n_keep),
+                                             _stream(stream))), "memosight_accept_static")

@@ -11,6 +11,8 @@
 // index -- the lowest-index-of-the-maximum convention with NaN treated as maximal.
 #include <limits.h>
 
+#include <mutex>
+
 #include "common.cuh"
 
 namespace {
@@ -148,6 +150,76 @@ extern "C" int32_t memosight_accept(const float* logits, int64_t ld_v, int32_t v
   cudaStream_t st = ms::as_stream(stream);
   const int n_chunks = chunks_of(vocab);
   Cand* part = static_cast<Cand*>(workspace);
+  if (total_rows > 0) {
+    const dim3 grid(static_cast<unsigned>(n_chunks) * static_cast<unsigned>(total_rows));
+    const bool vec = ms::aligned16(logits) && (ld_v % 4 == 0);
+    if (vec)
+      argmax_chunks_kernel<true><<<grid, kThreads, 0, st>>>(logits, ld_v, vocab, n_chunks, part);
+    else
+      argmax_chunks_kernel<false><<<grid, kThreads, 0, st>>>(logits, ld_v, vocab, n_chunks, part);
+    MS_LAUNCH_CHECK();
+  }
+  accept_rows_kernel<<<(batch + 3) / 4, 128, 0, st>>>(part, n_chunks, row_off, batch, draft,
+                                                      argmax_out, n_match, n_keep);
+  MS_LAUNCH_CHECK();
+  return MS_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Accept without any allocation by anyone.
+//
+// Some callers cannot obtain device memory at the moment they need an accept: code that runs
+// inside a memory-frozen serving loop (every byte was handed out at start-up and the allocator is
+// locked), plug-ins that are given tensors but no allocator handle, or hosts where cudaMalloc
+// would synchronise the device in the middle of a latency-critical step.  For them the per-chunk
+// candidates of pass 1 live in a fixed array inside the library image instead of a caller
+// workspace.  Every GPU that loads the library carries the array (512 KB) until the process exits.
+namespace {
+
+constexpr int kStaticMaxPartials = MS_ACCEPT_STATIC_MAX_PARTIALS;
+static_assert(kStaticMaxPartials == 65536, "keep the header's limit and the array in step");
+
+static __device__ __align__(256) unsigned char g_accept_scratch[kStaticMaxPartials * sizeof(Cand)];
+
+// In host code `g_accept_scratch` is only a handle for the runtime, not an address a kernel may
+// dereference: the device address is looked up once per device, with that device current.
+int32_t static_scratch_address(Cand** out) {
+  static std::mutex mu;
+  static Cand* addr[64] = {nullptr};
+  int dev = 0;
+  MS_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return MS_ERR_UNSUPPORTED_SHAPE;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!addr[dev]) {
+    void* p = nullptr;
+    MS_CUDA_TRY(cudaGetSymbolAddress(&p, g_accept_scratch));
+    if (!p) return ms::cuda_status(cudaErrorInvalidSymbol);
+    addr[dev] = static_cast<Cand*>(p);
+  }
+  *out = addr[dev];
+  return MS_OK;
+}
+
+}  // namespace
+
+extern "C" int32_t memosight_accept_static(const float* logits, int64_t ld_v, int32_t vocab,
+                                           const int32_t* row_off, int32_t batch,
+                                           int32_t total_rows, const int32_t* draft,
+                                           int32_t* argmax_out, int32_t* n_match, int32_t* n_keep,
+                                           memosight_stream_t stream) {
+  if (batch < 0 || total_rows < 0 || vocab < 1 || ld_v < vocab) return MS_ERR_INVALID_ARG;
+  if (batch == 0) return total_rows == 0 ? MS_OK : MS_ERR_INVALID_ARG;
+  if (!row_off || !n_match) return MS_ERR_INVALID_ARG;
+  if (total_rows > 0 && (!logits || !draft || !argmax_out)) return MS_ERR_INVALID_ARG;
+  const int n_chunks = chunks_of(vocab);
+  // the fixed array holds one candidate per (row, chunk): refuse anything larger, loudly
+  if (static_cast<int64_t>(total_rows) * n_chunks > kStaticMaxPartials) return MS_ERR_UNSUPPORTED_SHAPE;
+  Cand* part = nullptr;
+  const int32_t rc = static_scratch_address(&part);
+  if (rc != MS_OK) return rc;
+  cudaStream_t st = ms::as_stream(stream);
+  // Nothing in the array has to start at zero: pass 1 writes every (row, chunk) entry that pass 2
+  // reads, so whatever an earlier call left behind is overwritten before it is looked at.
   if (total_rows > 0) {
     const dim3 grid(static_cast<unsigned>(n_chunks) * static_cast<unsigned>(total_rows));
     const bool vec = ms::aligned16(logits) && (ld_v % 4 == 0);
