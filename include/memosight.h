@@ -122,7 +122,7 @@ typedef struct memosight_attn_params {
   int32_t batch;             /* B >= 0                                                         */
   int32_t n_q_heads;         /* H_q, multiple of n_kv_heads                                    */
   int32_t n_kv_heads;        /* H_kv                                                           */
-  int32_t head_dim;          /* D: 64 or 128 on the tensor-core path; any multiple of 32 up to
+  int32_t head_dim;          /* D: 64 or 128 on the tensor-core paths; any multiple of 32 up to
                                 256 on the general path                                        */
   const void* k_cache;       /* device bf16, one layer: [H_kv][n_slots][D], post-RoPE          */
   const void* v_cache;       /* device bf16, same layout                                       */
@@ -155,11 +155,24 @@ MS_API size_t memosight_attn_workspace_bytes(int32_t batch, int32_t n_q_heads, i
 
 /* Queues the attention of one layer (split-KV pass + log-sum-exp merge).
  * Limits: n_q_heads/n_kv_heads <= 16; max_nq <= 16; batch <= 8192 per call.
- * Blocks with max_nq * (H_q/H_kv) <= 64 and D in {64,128} take the tensor-core
- * path; anything else inside the limits takes the slower general path.
+ * Blocks with max_nq * (H_q/H_kv) <= 128 and D in {64,128} take a tensor-core
+ * path (mma.sync up to 32 packed rows, tcgen05 above); anything else inside the
+ * limits takes the slower general path.
  * The workspace may be reused by the next call on the same stream; two calls
  * that overlap on the GPU need two workspaces. */
 MS_API int32_t memosight_attn_step(const memosight_attn_params* params, memosight_stream_t stream);
+
+/* Diagnostic switch: which kernel memosight_attn_step uses from now on, process-wide.
+ * MS_ATTN_PATH_AUTO (the default) picks by shape: the mma.sync kernel up to 32 packed rows
+ * (max_nq * H_q/H_kv), the tcgen05 kernel up to 128, the general kernel otherwise.  Forcing a
+ * path that does not cover a shape falls back to the automatic choice for that call.  Returns
+ * the previous setting, or MS_ERR_INVALID_ARG.  Results of all paths agree within the
+ * tolerance of bf16 inputs with fp32 accumulation; the switch exists for tests and timing. */
+#define MS_ATTN_PATH_AUTO 0
+#define MS_ATTN_PATH_MMA_SYNC 1
+#define MS_ATTN_PATH_TCGEN05 2
+#define MS_ATTN_PATH_GENERAL 3
+MS_API int32_t memosight_attn_set_path(int32_t path);
 
 /* Synchronises `stream` and returns MS_OK, or MS_ERR_DEVICE_TIMEOUT if a kernel
  * of the last memosight_attn_step on this workspace gave up on a bounded wait

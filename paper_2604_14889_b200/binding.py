@@ -26,6 +26,11 @@ MS_ERR_ALIGNMENT = -4
 MS_ERR_CUDA = -5
 MS_ERR_DEVICE_TIMEOUT = -6
 
+MS_ATTN_PATH_AUTO = 0
+MS_ATTN_PATH_MMA_SYNC = 1
+MS_ATTN_PATH_TCGEN05 = 2
+MS_ATTN_PATH_GENERAL = 3
+
 MS_ROPE_NEOX = 0
 MS_ROPE_INTERLEAVED = 1
 MS_POS_HALF_UNITS = 2
@@ -105,6 +110,8 @@ def lib() -> C.CDLL:
         L.memosight_attn_workspace_bytes.argtypes = [C.c_int32] * 6
         L.memosight_attn_step.restype = C.c_int32
         L.memosight_attn_step.argtypes = [C.POINTER(AttnParams), C.c_void_p]
+        L.memosight_attn_set_path.restype = C.c_int32
+        L.memosight_attn_set_path.argtypes = [C.c_int32]
         L.memosight_attn_status.restype = C.c_int32
         L.memosight_attn_status.argtypes = [C.c_void_p, C.c_void_p]
         L.memosight_kv_compact.restype = C.c_int32
@@ -234,6 +241,14 @@ def memosight_attn_step(params: Optional[AttnParams] = None, stream=None, **fiel
 
 def memosight_step_host(params: StepHostParams, stream=None) -> None:
     _check(int(lib().memosight_step_host(C.byref(params), _stream(stream))), "memosight_step_host")
+
+
+def memosight_attn_set_path(path: int) -> int:
+    """Selects the attention kernel (MS_ATTN_PATH_*); returns the previous setting."""
+    rc = int(lib().memosight_attn_set_path(int(path)))
+    if rc < 0:
+        raise MemosightError(rc, "memosight_attn_set_path")
+    return rc
 
 
 def memosight_attn_status(workspace, stream=None) -> int:

@@ -4,13 +4,39 @@
 
 #include "attn_internal.cuh"
 
+#include <atomic>
+
 namespace {
 
+std::atomic<int32_t> g_forced_path{MS_ATTN_PATH_AUTO};
+
+bool mma_shape(int D, int G, int max_nq) { return (D == 64 || D == 128) && max_nq * G <= 64; }
+
+// Either tensor-core path: both use the per-CTA partial slots of the split-KV workspace.
 bool fast_path_shape(int D, int G, int max_nq) {
-  return (D == 64 || D == 128) && max_nq * G <= 64;
+  return mma_shape(D, G, max_nq) || ms::attn_umma_supports(D, G, max_nq);
+}
+
+// Which kernel serves a shape: blocks of up to 32 packed rows stream fastest through the
+// mma.sync kernel; above that every K/V byte would be re-read from shared memory once per
+// 16-row block, so the tcgen05 kernel (operands straight from shared memory) takes over.
+int32_t pick_path(int D, int G, int max_nq) {
+  const int32_t forced = g_forced_path.load(std::memory_order_relaxed);
+  const bool mma_ok = mma_shape(D, G, max_nq), umma_ok = ms::attn_umma_supports(D, G, max_nq);
+  if (forced == MS_ATTN_PATH_MMA_SYNC && mma_ok) return forced;
+  if (forced == MS_ATTN_PATH_TCGEN05 && umma_ok) return forced;
+  if (forced == MS_ATTN_PATH_GENERAL) return forced;
+  if (mma_ok && (max_nq * G <= 32 || !umma_ok)) return MS_ATTN_PATH_MMA_SYNC;
+  if (umma_ok) return MS_ATTN_PATH_TCGEN05;
+  return MS_ATTN_PATH_GENERAL;
 }
 
 }  // namespace
+
+extern "C" int32_t memosight_attn_set_path(int32_t path) {
+  if (path < MS_ATTN_PATH_AUTO || path > MS_ATTN_PATH_GENERAL) return MS_ERR_INVALID_ARG;
+  return g_forced_path.exchange(path, std::memory_order_relaxed);
+}
 
 extern "C" size_t memosight_attn_workspace_bytes(int32_t batch, int32_t n_q_heads,
                                                  int32_t n_kv_heads, int32_t head_dim,
@@ -76,8 +102,10 @@ extern "C" int32_t memosight_attn_step(const memosight_attn_params* p, memosight
 
   cudaStream_t st = ms::as_stream(stream);
   // An empty cache tensor still needs a valid address for the tile descriptors.
-  if (fast_path_shape(a.D, G, a.max_nq) && a.k_cache && a.v_cache && a.n_slots >= 1)
-    return ms::launch_attn_mma(a, st);
+  const int32_t path = (a.k_cache && a.v_cache && a.n_slots >= 1) ? pick_path(a.D, G, a.max_nq)
+                                                                   : MS_ATTN_PATH_GENERAL;
+  if (path == MS_ATTN_PATH_MMA_SYNC) return ms::launch_attn_mma(a, st);
+  if (path == MS_ATTN_PATH_TCGEN05) return ms::launch_attn_umma(a, st);
   return ms::launch_attn_simt(a, st);
 }
 

@@ -41,4 +41,9 @@ size_t attn_mma_workspace_bytes(int D, int rows_pad, int n_ctas);
 int32_t launch_attn_mma(const AttnArgs& a, cudaStream_t st);
 int attn_mma_grid();   // persistent CTAs the split kernel launches on this device
 
+// tcgen05 split-KV path (operands from shared memory, accumulators in tensor memory):
+// up to 128 packed rows per KV head; same workspace layout and merge as the path above.
+bool attn_umma_supports(int D, int G, int max_nq);
+int32_t launch_attn_umma(const AttnArgs& a, cudaStream_t st);
+
 }  // namespace ms
