@@ -61,7 +61,7 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample-seqs", type=int, default=32)
-    ap.add_argument("--attn-path", default="auto", choices=["auto", "mma_sync", "tcgen05"],
+    ap.add_argument("--attn-path", default="auto", choices=["auto", "mma_sync", "tcgen05", "tcgen05_keys"],
                     help="attention kernel: by shape (default), or forced for A/B timing")
     return ap.parse_args()
 
@@ -295,7 +295,8 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     ms.memosight_attn_set_path({"auto": ms.MS_ATTN_PATH_AUTO, "mma_sync": ms.MS_ATTN_PATH_MMA_SYNC,
-                                "tcgen05": ms.MS_ATTN_PATH_TCGEN05}[args.attn_path])
+                                "tcgen05": ms.MS_ATTN_PATH_TCGEN05,
+                                "tcgen05_keys": ms.MS_ATTN_PATH_TCGEN05_KEYS}[args.attn_path])
     K, W = args.steps, max(args.warmup, 3)
     cfg0 = synth.sweep(args.batch, args.d, args.kv_len, True)
     n_e2e = 0 if args.no_e2e else max(1, min(args.e2e_steps, K))
@@ -392,7 +393,10 @@ def main():
     peak, peak_kind = peak_hbm()
     rows = nq * (Hq // Hkv)
     use_umma = args.attn_path == "tcgen05" or (args.attn_path == "auto" and rows > 32)
-    kernel_name = "attn_umma_kernel<128>" if use_umma else f"attn_split_kernel<128,{1 if rows <= 16 else 2 if rows <= 32 else 4}>"
+    if args.attn_path == "tcgen05_keys":
+        kernel_name = f"attn_umma_t_kernel<{(rows + 15) // 16 * 16}>"
+    else:
+        kernel_name = "attn_umma_kernel<128>" if use_umma else f"attn_split_kernel<128,{1 if rows <= 16 else 2 if rows <= 32 else 4}>"
     roofline = {"bound": "hbm", "kernel": kernel_name, "achieved": achieved, "peak": peak,
                 "peak_source": f"{peak_kind} copy bandwidth", "unit": "GB/s", "frac": achieved / peak,
                 "frac_of_nominal_8000": achieved / 8000.0, "avg_launch_ms": split_avg_ms,

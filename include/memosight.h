@@ -172,6 +172,7 @@ MS_API int32_t memosight_attn_step(const memosight_attn_params* params, memosigh
 #define MS_ATTN_PATH_MMA_SYNC 1
 #define MS_ATTN_PATH_TCGEN05 2
 #define MS_ATTN_PATH_GENERAL 3
+#define MS_ATTN_PATH_TCGEN05_KEYS 4   /* tcgen05 with the keys on the accumulator lanes; <= 64 rows, D 128 */
 MS_API int32_t memosight_attn_set_path(int32_t path);
 
 /* Synchronises `stream` and returns MS_OK, or MS_ERR_DEVICE_TIMEOUT if a kernel

@@ -30,6 +30,7 @@ MS_ATTN_PATH_AUTO = 0
 MS_ATTN_PATH_MMA_SYNC = 1
 MS_ATTN_PATH_TCGEN05 = 2
 MS_ATTN_PATH_GENERAL = 3
+MS_ATTN_PATH_TCGEN05_KEYS = 4
 
 MS_ROPE_NEOX = 0
 MS_ROPE_INTERLEAVED = 1

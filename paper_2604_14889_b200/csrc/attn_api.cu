@@ -23,8 +23,10 @@ bool fast_path_shape(int D, int G, int max_nq) {
 int32_t pick_path(int D, int G, int max_nq) {
   const int32_t forced = g_forced_path.load(std::memory_order_relaxed);
   const bool mma_ok = mma_shape(D, G, max_nq), umma_ok = ms::attn_umma_supports(D, G, max_nq);
+  const bool umma_t_ok = ms::attn_umma_t_supports(D, G, max_nq);
   if (forced == MS_ATTN_PATH_MMA_SYNC && mma_ok) return forced;
   if (forced == MS_ATTN_PATH_TCGEN05 && umma_ok) return forced;
+  if (forced == MS_ATTN_PATH_TCGEN05_KEYS && umma_t_ok) return forced;
   if (forced == MS_ATTN_PATH_GENERAL) return forced;
   if (mma_ok && (max_nq * G <= 32 || !umma_ok)) return MS_ATTN_PATH_MMA_SYNC;
   if (umma_ok) return MS_ATTN_PATH_TCGEN05;
@@ -34,7 +36,7 @@ int32_t pick_path(int D, int G, int max_nq) {
 }  // namespace
 
 extern "C" int32_t memosight_attn_set_path(int32_t path) {
-  if (path < MS_ATTN_PATH_AUTO || path > MS_ATTN_PATH_GENERAL) return MS_ERR_INVALID_ARG;
+  if (path < MS_ATTN_PATH_AUTO || path > MS_ATTN_PATH_TCGEN05_KEYS) return MS_ERR_INVALID_ARG;
   return g_forced_path.exchange(path, std::memory_order_relaxed);
 }
 
@@ -106,6 +108,7 @@ extern "C" int32_t memosight_attn_step(const memosight_attn_params* p, memosight
                                                                    : MS_ATTN_PATH_GENERAL;
   if (path == MS_ATTN_PATH_MMA_SYNC) return ms::launch_attn_mma(a, st);
   if (path == MS_ATTN_PATH_TCGEN05) return ms::launch_attn_umma(a, st);
+  if (path == MS_ATTN_PATH_TCGEN05_KEYS) return ms::launch_attn_umma_t(a, st);
   return ms::launch_attn_simt(a, st);
 }
 

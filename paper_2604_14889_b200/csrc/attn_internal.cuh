@@ -46,4 +46,9 @@ int attn_mma_grid();   // persistent CTAs the split kernel launches on this devi
 bool attn_umma_supports(int D, int G, int max_nq);
 int32_t launch_attn_umma(const AttnArgs& a, cudaStream_t st);
 
+// tcgen05 path with the tile's keys on the tensor-memory lanes (the transposed products):
+// blocks of up to 64 packed rows, head_dim 128.
+bool attn_umma_t_supports(int D, int G, int max_nq);
+int32_t launch_attn_umma_t(const AttnArgs& a, cudaStream_t st);
+
 }  // namespace ms

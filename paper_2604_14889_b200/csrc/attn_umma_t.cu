@@ -1,0 +1,583 @@
+// Keys-on-lanes tcgen05 split-KV path of the MemoSight step attention (sm_100a).
+//
+// The step block of MemoSight (paper Sec. 2.1.1) is small -- n_q*G = 8..64 packed
+// query rows per KV head -- while a K/V tile is 128 keys.  Putting the query rows
+// on the 128 rows of the MMA tile would leave most tensor-memory lanes (and with
+// them most of the four SM sub-partitions, each of which can only reach its own
+// 32 lanes) idle in the softmax.  This kernel therefore computes the transposed
+// problem, the tile's 128 keys on the lanes:
+//     S^T[key][row] = K_tile (A, K-major)   x  Q^T (B = Q, K-major)      N = rows padded to 16
+//     O^T[d][row]  += V_tile^T (A, MN-major) x  P^T (B, MN-major)         M = D = 128
+// so that every softmax thread owns one key of the tile and touches only as many
+// score columns as there are query rows: the softmax cost follows the block size
+// and all four sub-partitions work on every tile.  The mask is then a per-thread
+// predicate (key index against the valid length; the (n_cand, anchor) rule on the
+// step-local tile).
+//
+// Row statistics need the keys of all lanes:
+//   * the reference maximum m_ref[row] is the exact row maximum of the unit's first
+//     tile (redux.sync.max per warp, combined through shared memory); later tiles
+//     are exponentiated against it unchanged.  Any shift is exact for a softmax as
+//     long as nothing overflows, so m_ref only moves when a score exceeds it by
+//     more than 2^48: the four softmax warps agree on that each tile through one
+//     mbarrier round, and then rescale O^T and the partial sums together (rare).
+//   * the row sums stay per thread (one partial per key lane and row) and are
+//     reduced across lanes once, at the end of the unit.
+// Roles, pipeline, schedule, workspace format and bounded waits are those of the
+// rows-on-lanes kernel (attn_umma.cu); head_dim is 128.
+#include "attn_umma_common.cuh"
+
+namespace ms {
+namespace {
+
+constexpr int kTThreads = 256;
+constexpr float kGrowLimit = 48.f;
+constexpr int kTMaxKv = 8;
+constexpr int kPBytes = kTile * 128;            // P^T tile: 128 keys x 64 columns of bf16
+constexpr int kKvBytes = kTile * 128 * 2;       // K or V tile, D = 128
+constexpr uint32_t kHalfStrideT = kTile * 128;  // bytes between the 64-column halves of a K/V tile
+
+enum : int {
+  kTbKvFull = 0, kTbKvEmpty = kTMaxKv, kTbQFull = 2 * kTMaxKv, kTbQEmpty = kTbQFull + 2,
+  kTbSFull = kTbQEmpty + 2, kTbPFull = kTbSFull + 2, kTbPvDone = kTbPFull + 2, kTbWg = kTbPvDone + 2,
+  kTbDrain = kTbWg + 1, kTbCount = kTbDrain + 1
+};
+// misc region behind the ring: barriers | scalars | m_ref[64] | red[4][64]
+constexpr int kMiscScalars = 256, kMiscMref = 512, kMiscRed = 768, kMiscBytes = 2048;
+static_assert(kTbCount * 8 <= kMiscScalars, "barriers overflow their slot");
+
+struct TLayout {
+  int rows_box;      // rows one Q box holds: G * max_nq
+  int q_half, q_bytes, n_kv;
+  int off_q, off_p, off_kv, off_misc, total;
+};
+
+// Sum of v[j] over the 32 lanes for 32 rows at once: lane L ends up with the total of row L.
+__device__ __forceinline__ float warp_sum_32rows(float (&t)[32], int lane) {
+#pragma unroll
+  for (int o = 16; o >= 1; o >>= 1) {
+    const bool up = (lane & o) != 0;
+#pragma unroll
+    for (int i = 0; i < o; ++i) {
+      const float send = up ? t[i] : t[i + o];
+      const float keep = up ? t[i + o] : t[i];
+      t[i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+    }
+  }
+  return t[0];
+}
+
+template <int NP>
+__global__ void __launch_bounds__(kTThreads, 1)
+attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
+                   const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_ks,
+                   const __grid_constant__ CUtensorMap map_vs, const __grid_constant__ CUtensorMap map_q,
+                   int rows_pad, const TLayout lay) {
+  constexpr int D = 128, HALVES = 2, KSTEPS_QK = D / 16;
+  constexpr int GROUPS = (NP + 31) / 32;
+  constexpr uint32_t kCols = NP <= 16 ? 64 : (NP <= 32 ? 128 : 256);   // S^T x2 and O^T, a power of two
+  constexpr uint32_t kColO = 2 * NP;
+  extern __shared__ __align__(1024) uint8_t smem[];
+  const uint32_t sb = smem_u32(smem);
+  const uint32_t bars = sb + lay.off_misc;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + lay.off_misc + kMiscScalars);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + lay.off_misc + kMiscScalars + 8);
+  volatile int* grow_flag = reinterpret_cast<volatile int*>(smem + lay.off_misc + kMiscScalars + 16);
+  float* s_mref = reinterpret_cast<float*>(smem + lay.off_misc + kMiscMref);
+  float* s_red = reinterpret_cast<float*>(smem + lay.off_misc + kMiscRed);
+  uint32_t* status = reinterpret_cast<uint32_t*>(a.workspace);
+  int* ws_pre = reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(a.workspace) + kWsHeaderBytes);
+  float* ws_slots = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(a.workspace) + kWsHeaderBytes +
+                                             ws_prefix_bytes());
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (sb & 1023u) {
+    if (threadIdx.x == 0) atomicExch(status, kTimeoutMagic + 1);
+    return;
+  }
+
+  // ---- schedule (the prefix lives where the buffers will be) ----
+  int* s_pre = reinterpret_cast<int*>(smem);
+  int* s_scratch = s_pre + a.B + 1;
+  build_tile_prefix(a, s_pre, s_scratch);
+  const long long n_tiles = static_cast<long long>(s_pre[a.B]) * a.H_kv;
+  const long long t0 = n_tiles * blockIdx.x / gridDim.x;
+  const long long t1 = n_tiles * (blockIdx.x + 1) / gridDim.x;
+  const int n_iter = static_cast<int>(t1 - t0);
+  if (blockIdx.x == 0) {
+    for (int i = threadIdx.x; i <= a.B; i += blockDim.x) ws_pre[i] = s_pre[i];
+  }
+  Walk w0;
+  w0.n_iter = 0;
+  if (n_iter > 0) {
+    int lo = 0, hi = a.B;
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (static_cast<long long>(s_pre[mid]) * a.H_kv <= t0) lo = mid; else hi = mid;
+    }
+    walk_init(a, w0, lo, t0 - static_cast<long long>(s_pre[lo]) * a.H_kv, n_iter);
+  }
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kTMaxKv; ++i) {
+      mbar_init(bars + 8 * (kTbKvFull + i), 1);
+      mbar_init(bars + 8 * (kTbKvEmpty + i), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bars + 8 * (kTbQFull + i), 1);
+      mbar_init(bars + 8 * (kTbQEmpty + i), 1);
+      mbar_init(bars + 8 * (kTbSFull + i), 1);
+      mbar_init(bars + 8 * (kTbPFull + i), 4);
+      mbar_init(bars + 8 * (kTbPvDone + i), 1);
+    }
+    mbar_init(bars + 8 * kTbWg, 4);
+    mbar_init(bars + 8 * kTbDrain, 1);
+    *abort_flag = 0;
+    *grow_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();   // the prefix has been consumed
+  // Rows of the Q buffers past the box are never loaded; as B rows they only feed the padded
+  // score columns, which must stay finite: clear them once.
+  {
+    const int pad_rows = NP - lay.rows_box;
+    for (int x = threadIdx.x; x < pad_rows * 2 * HALVES * 8; x += blockDim.x) {
+      const int c = x & 7, rest = x >> 3;
+      const int rr = lay.rows_box + rest % pad_rows, buf_half = rest / pad_rows;   // 0..3
+      const uint32_t addr = sb + lay.off_q + (buf_half >> 1) * lay.q_bytes + (buf_half & 1) * lay.q_half +
+                            rr * 128 + (c << 4);
+      asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(addr), "r"(0u) : "memory");
+    }
+    fence_async_smem();
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                     smem_u32(tmem_slot)), "r"(kCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  if (warp == 0 && lane == 0 && n_iter > 0) {
+    // =========================== TMA producer ===========================
+    Walk w = w0;
+    bool ok = true;
+    int uses = 0, pieces = 0;
+    while (w.it < n_iter) {
+      walk_tile(a, w);
+      if (w.first) {
+        const int qb = w.piece_idx & 1;
+        if (!mbar_wait(bars + 8 * (kTbQEmpty + qb), ((w.piece_idx >> 1) & 1) ^ 1, abort_flag, status)) {
+          ok = false;
+          break;
+        }
+        fence_async_smem();
+        const uint32_t bar = bars + 8 * (kTbQFull + qb);
+        mbar_arrive_expect_tx(bar, static_cast<uint32_t>(HALVES * lay.rows_box * 128));
+#pragma unroll
+        for (int hf = 0; hf < HALVES; ++hf)
+          tma_load_3d(sb + lay.off_q + qb * lay.q_bytes + hf * lay.q_half, &map_q, bar, hf * 64, w.h * a.G,
+                      w.r0);
+        ++pieces;
+      }
+#pragma unroll 1
+      for (int kv = 0; kv < 2; ++kv) {
+        const int use = 2 * w.it + kv;
+        const int buf = use % lay.n_kv;
+        if (!mbar_wait(bars + 8 * (kTbKvEmpty + buf), ((use / lay.n_kv) & 1) ^ 1, abort_flag, status)) {
+          ok = false;
+          break;
+        }
+        fence_async_smem();
+        const uint32_t dst = sb + lay.off_kv + buf * kKvBytes;
+        const uint32_t bar = bars + 8 * (kTbKvFull + buf);
+        if (w.is_step) {
+          mbar_arrive_expect_tx(bar, static_cast<uint32_t>(HALVES * kMaxNq * 128));
+#pragma unroll
+          for (int hf = 0; hf < HALVES; ++hf)
+            tma_load_3d(dst + hf * kHalfStrideT, kv ? &map_vs : &map_ks, bar, hf * 64, w.h, w.r0);
+        } else {
+          mbar_arrive_expect_tx(bar, static_cast<uint32_t>(kKvBytes));
+          const int y = static_cast<int>(w.slot_off) + w.ti * kTile;
+#pragma unroll
+          for (int hf = 0; hf < HALVES; ++hf)
+            tma_load_3d(dst + hf * kHalfStrideT, kv ? &map_v : &map_k, bar, hf * 64, y, w.h);
+        }
+        ++uses;
+      }
+      if (!ok) break;
+      walk_next(a, w);
+    }
+    // Drain: every copy issued here must have landed before the CTA may exit.
+    for (int u = uses > lay.n_kv ? uses - lay.n_kv : 0; u < uses; ++u)
+      (void)mbar_wait(bars + 8 * (kTbKvFull + u % lay.n_kv), (u / lay.n_kv) & 1, abort_flag, status);
+    for (int p = pieces > 2 ? pieces - 2 : 0; p < pieces; ++p)
+      (void)mbar_wait(bars + 8 * (kTbQFull + (p & 1)), (p >> 1) & 1, abort_flag, status);
+  } else if (warp == 1 && lane == 0 && n_iter > 0) {
+    // =========================== MMA issuer ===========================
+    const uint32_t idesc_qk = instr_desc(NP, 0, 0);     // A = K tile (K-major), B = Q (K-major)
+    const uint32_t idesc_pv = instr_desc(NP, 1, 1);     // A = V tile^T (MN-major), B = P^T (MN-major)
+    Walk wq = w0, wp = w0;
+    bool ok = true;
+    auto issue_qk = [&]() -> bool {
+      walk_tile(a, wq);
+      const int it = wq.it, qb = wq.piece_idx & 1;
+      if (wq.first &&
+          !mbar_wait(bars + 8 * (kTbQFull + qb), (wq.piece_idx >> 1) & 1, abort_flag, status))
+        return false;
+      const int use = 2 * it, buf = use % lay.n_kv;
+      if (!mbar_wait(bars + 8 * (kTbKvFull + buf), (use / lay.n_kv) & 1, abort_flag, status)) return false;
+      tc_fence_after();
+      const uint32_t qa = sb + lay.off_q + qb * lay.q_bytes;
+      const uint32_t ka = sb + lay.off_kv + buf * kKvBytes;
+      const uint32_t d_s = tmem + (it & 1) * NP;
+#pragma unroll
+      for (int ks = 0; ks < KSTEPS_QK; ++ks) {
+        const uint32_t koff = (ks >> 2) * kHalfStrideT + (ks & 3) * 32;
+        const uint32_t qoff = (ks >> 2) * lay.q_half + (ks & 3) * 32;
+        umma_bf16(d_s, smem_desc(ka + koff, 16), smem_desc(qa + qoff, 16), idesc_qk, ks > 0);
+      }
+      umma_commit(bars + 8 * (kTbKvEmpty + buf));
+      umma_commit(bars + 8 * (kTbSFull + (it & 1)));
+      if (wq.last) umma_commit(bars + 8 * (kTbQEmpty + qb));
+      walk_next(a, wq);
+      return true;
+    };
+    ok = issue_qk();
+    while (ok && wp.it < n_iter) {
+      if (wq.it < n_iter && !issue_qk()) { ok = false; break; }
+      walk_tile(a, wp);
+      const int it = wp.it;
+      const int use = 2 * it + 1, buf = use % lay.n_kv;
+      if (!mbar_wait(bars + 8 * (kTbPFull + (it & 1)), (it >> 1) & 1, abort_flag, status) ||
+          !mbar_wait(bars + 8 * (kTbKvFull + buf), (use / lay.n_kv) & 1, abort_flag, status)) {
+        ok = false;
+        break;
+      }
+      tc_fence_after();
+      const uint32_t pa = sb + lay.off_p + (it & 1) * kPBytes;
+      const uint32_t va = sb + lay.off_kv + buf * kKvBytes;
+      const int ksteps = wp.is_step ? 1 : (wp.nvalid + 15) >> 4;
+#pragma unroll 1
+      for (int j = 0; j < ksteps; ++j)
+        umma_bf16(tmem + kColO, smem_desc(va + j * 2048, kHalfStrideT), smem_desc(pa + j * 2048, kHalfStrideT),
+                  idesc_pv, !(wp.first && j == 0));
+      umma_commit(bars + 8 * (kTbKvEmpty + buf));
+      umma_commit(bars + 8 * (kTbPvDone + (it & 1)));
+      walk_next(a, wp);
+    }
+    if (!ok) {
+      umma_commit(bars + 8 * kTbDrain);
+      const unsigned long long t_begin = global_ns();
+      while (!mbar_try_wait(bars + 8 * kTbDrain, 0) && global_ns() - t_begin < kWaitLimitNs) {
+      }
+    }
+  } else if (warp >= 4 && n_iter > 0) {
+    // =========================== softmax warps: thread = key of the tile ===========================
+    const int quad = warp - 4;
+    const int t = quad * 32 + lane;                        // key index in the tile = TMEM lane
+    const uint32_t lane_addr = tmem + (static_cast<uint32_t>(quad * 32) << 16);
+    const uint32_t tx = t & 7;
+    float* red_w = s_red + quad * 64;
+    Walk w = w0;
+    float lsum[NP];
+    uint32_t wg_phase = 0;
+    bool ok = true;
+    auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {
+      return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, status));
+    };
+    // bounded barrier of the four softmax warps (also publishes their shared-memory writes)
+    auto wg_sync = [&]() -> bool {
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bars + 8 * kTbWg);
+      const bool good = wait_all(bars + 8 * kTbWg, wg_phase & 1);
+      ++wg_phase;
+      return good;
+    };
+    while (ok && w.it < n_iter) {
+      walk_tile(a, w);
+      const int it = w.it, pb = it & 1;
+      if (!wait_all(bars + 8 * (kTbSFull + pb), (it >> 1) & 1)) { ok = false; break; }
+      if (it >= 2 && !wait_all(bars + 8 * (kTbPvDone + pb), ((it >> 1) - 1) & 1)) { ok = false; break; }
+      tc_fence_after();
+      const int nv = w.nvalid;
+      if (w.is_step || nv < kTile) {
+        // V rows past the valid keys hold foreign or stale bytes; their P is 0 but 0 * NaN is NaN:
+        // clear the rows of the last 16-key step that the PV product still reads
+        const int use = 2 * it + 1, buf = use % lay.n_kv;
+        if (!wait_all(bars + 8 * (kTbKvFull + buf), (use / lay.n_kv) & 1)) { ok = false; break; }
+        const uint32_t va = sb + lay.off_kv + buf * kKvBytes;
+        const int n_rows = ((nv + 15) & ~15) - nv;
+        for (int x = t; x < n_rows * HALVES * 8; x += 128) {
+          const int rr = nv + x / (HALVES * 8), cc = x % (HALVES * 8);
+          const uint32_t addr = va + (cc >> 3) * kHalfStrideT + rr * 128 + ((cc & 7) << 4);
+          asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(addr), "r"(0u) : "memory");
+        }
+      }
+      const bool key_ok = t < nv;
+      const uint32_t s_addr = lane_addr + pb * NP;
+
+      // scores of this key against every row; invisible pairs become -inf
+      float v[NP];
+      auto load_scores = [&]() {
+        uint32_t raw[NP];
+#pragma unroll
+        for (int c = 0; c < NP / 16; ++c) tmem_ld16(s_addr + c * 16, raw + c * 16);
+#pragma unroll
+        for (int c = 0; c < NP / 16; ++c) tmem_ld_wait16(raw + c * 16);
+        if (!w.is_step) {
+#pragma unroll
+          for (int j = 0; j < NP; ++j) v[j] = key_ok ? __uint_as_float(raw[j]) : -INFINITY;
+        } else {
+          int i = 0, g = 0;
+#pragma unroll
+          for (int j = 0; j < NP; ++j) {
+            bool vis = false;
+            if (key_ok && i < w.n_q) {
+              const int anc = (i < w.n_c) ? i : (a.anchor ? a.anchor[w.r0 + i] : w.n_c);
+              vis = step_key_visible(i, t, w.n_c, anc);
+            }
+            v[j] = vis ? __uint_as_float(raw[j]) : -INFINITY;
+            if (++g == a.G) { g = 0; ++i; }
+          }
+        }
+      };
+      // exact maximum over the tile's keys of every row -> red[warp][row]
+      auto reduce_row_max = [&]() {
+        float keep[GROUPS];
+#pragma unroll
+        for (int g = 0; g < GROUPS; ++g) keep[g] = -INFINITY;
+#pragma unroll
+        for (int j = 0; j < NP; ++j) {
+          const float r = warp_max_f32(v[j]);
+          if (lane == (j & 31)) keep[j >> 5] = r;
+        }
+#pragma unroll
+        for (int g = 0; g < GROUPS; ++g) red_w[g * 32 + lane] = keep[g];
+      };
+      load_scores();
+
+      if (w.piece_j == 0) {
+        // new unit: the reference maximum of each row is the exact maximum of this first tile
+        reduce_row_max();
+        if (!wg_sync()) { ok = false; break; }
+        if (t < NP) {
+          const float m = fmaxf(fmaxf(s_red[t], s_red[64 + t]), fmaxf(s_red[128 + t], s_red[192 + t]));
+          s_mref[t] = (m == -INFINITY) ? 0.f : m * a.scale_log2;
+        }
+        if (!wg_sync()) { ok = false; break; }
+#pragma unroll
+        for (int j = 0; j < NP; ++j) lsum[j] = 0.f;
+      }
+
+      // x = s * scale - m_ref (log2 units)
+      float tmaxx = -INFINITY;
+#pragma unroll
+      for (int j4 = 0; j4 < NP / 4; ++j4) {
+        const float4 m4 = *reinterpret_cast<const float4*>(s_mref + 4 * j4);
+        v[4 * j4 + 0] = fmaf(v[4 * j4 + 0], a.scale_log2, -m4.x);
+        v[4 * j4 + 1] = fmaf(v[4 * j4 + 1], a.scale_log2, -m4.y);
+        v[4 * j4 + 2] = fmaf(v[4 * j4 + 2], a.scale_log2, -m4.z);
+        v[4 * j4 + 3] = fmaf(v[4 * j4 + 3], a.scale_log2, -m4.w);
+        tmaxx = fmaxf(tmaxx, fmaxf(fmaxf(v[4 * j4], v[4 * j4 + 1]), fmaxf(v[4 * j4 + 2], v[4 * j4 + 3])));
+      }
+      // the four warps agree on whether any score outgrew its reference (tile index as the token)
+      if (w.piece_j > 0 && __any_sync(0xffffffffu, tmaxx > kGrowLimit) && lane == 0) *grow_flag = it + 1;
+      if (!wg_sync()) { ok = false; break; }
+      if (*grow_flag == it + 1) {
+        // ---- rare: move the references up, rescale O^T and the partial sums, redo x ----
+        load_scores();
+        reduce_row_max();
+        if (!wg_sync()) { ok = false; break; }
+        float alpha[NP];
+#pragma unroll
+        for (int j = 0; j < NP; ++j) {
+          const float m = fmaxf(fmaxf(s_red[j], s_red[64 + j]), fmaxf(s_red[128 + j], s_red[192 + j]));
+          const float m_old = s_mref[j];
+          const float m_new = (m == -INFINITY) ? m_old : fmaxf(m_old, m * a.scale_log2);
+          alpha[j] = ex2(m_old - m_new);
+          lsum[j] *= alpha[j];
+          v[j] = fmaf(v[j], a.scale_log2, -m_new);
+        }
+        if (!wg_sync()) { ok = false; break; }          // everyone has read the old references
+        if (t < NP) {
+          const float m = fmaxf(fmaxf(s_red[t], s_red[64 + t]), fmaxf(s_red[128 + t], s_red[192 + t]));
+          if (m != -INFINITY) s_mref[t] = fmaxf(s_mref[t], m * a.scale_log2);
+        }
+        // all PV products issued so far are complete before O^T is touched
+        if (!wait_all(bars + 8 * (kTbPvDone + ((it - 1) & 1)), ((it - 1) >> 1) & 1)) { ok = false; break; }
+        tc_fence_after();
+        {
+          uint32_t o[NP];
+#pragma unroll
+          for (int c = 0; c < NP / 16; ++c) tmem_ld16(lane_addr + kColO + c * 16, o + c * 16);
+#pragma unroll
+          for (int c = 0; c < NP / 16; ++c) tmem_ld_wait16(o + c * 16);
+#pragma unroll
+          for (int j = 0; j < NP; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha[j]);
+#pragma unroll
+          for (int c = 0; c < NP / 16; ++c) tmem_st16(lane_addr + kColO + c * 16, o + c * 16);
+          asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+        }
+        if (!wg_sync()) { ok = false; break; }          // new references visible to later tiles
+      }
+
+      // p = 2^x as bf16 into this key's row of the P^T tile; partial row sums stay in registers
+      {
+        const uint32_t p_row = sb + lay.off_p + pb * kPBytes + t * 128;
+#pragma unroll
+        for (int c = 0; c < NP / 8; ++c) {
+          float p[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            p[e] = ex2(v[c * 8 + e]);
+            lsum[c * 8 + e] += p[e];
+          }
+          const uint32_t addr = p_row + ((c ^ tx) << 4);
+          asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(pack2(p[0], p[1])),
+                       "r"(pack2(p[2], p[3])), "r"(pack2(p[4], p[5])), "r"(pack2(p[6], p[7]))
+                       : "memory");
+        }
+      }
+      fence_async_smem();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bars + 8 * (kTbPFull + pb));
+
+      if (w.last) {
+        // ---- end of the unit (or of this CTA's part of it) ----
+        // row sums: over the 32 lanes of each warp, then over the four warps
+#pragma unroll
+        for (int g = 0; g < GROUPS; ++g) {
+          float tsum[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) tsum[i] = (g * 32 + i < NP) ? lsum[(g * 32 + i < NP) ? g * 32 + i : 0] : 0.f;
+          red_w[g * 32 + lane] = warp_sum_32rows(tsum, lane);
+        }
+        if (!wg_sync()) { ok = false; break; }
+        const int rows = w.n_q * a.G;
+        float l_row[NP];
+#pragma unroll
+        for (int j = 0; j < NP; ++j) l_row[j] = (s_red[j] + s_red[64 + j]) + (s_red[128 + j] + s_red[192 + j]);
+        const float m_mine = (t < NP) ? s_mref[t] : 0.f;
+        if (!wg_sync()) { ok = false; break; }          // red and m_ref may be reused from here on
+        if (!wait_all(bars + 8 * (kTbPvDone + pb), (it >> 1) & 1)) { ok = false; break; }
+        tc_fence_after();
+        uint32_t o[NP];
+#pragma unroll
+        for (int c = 0; c < NP / 16; ++c) tmem_ld16(lane_addr + kColO + c * 16, o + c * 16);
+#pragma unroll
+        for (int c = 0; c < NP / 16; ++c) tmem_ld_wait16(o + c * 16);
+        // thread t holds element d = t of every row
+        if (w.slot < 0) {
+          int i = 0, g = 0;
+#pragma unroll
+          for (int j = 0; j < NP; ++j) {
+            if (j < rows) {
+              const int64_t orow = static_cast<int64_t>(w.r0 + i) * a.H_q + w.h * a.G + g;
+              a.out[orow * D + t] = __float2bfloat16_rn(__uint_as_float(o[j]) / l_row[j]);
+              if (a.lse && t == j) a.lse[orow] = (m_mine + log2f(l_row[j])) * 0.69314718055994531f;
+            }
+            if (++g == a.G) { g = 0; ++i; }
+          }
+        } else {
+          float* slot = ws_slots + static_cast<size_t>(w.slot) * ws_slot_floats(D, rows_pad);
+          float* sm = slot + static_cast<size_t>(rows_pad) * D;
+#pragma unroll
+          for (int j = 0; j < NP; ++j) {
+            if (j < rows) {
+              slot[static_cast<size_t>(j) * D + t] = __uint_as_float(o[j]);
+              if (t == j) {
+                sm[j] = m_mine;
+                sm[rows_pad + j] = l_row[j];
+              }
+            }
+          }
+        }
+        tc_fence_before();   // the reads of O^T are ordered before the next unit's first PV product
+      }
+      walk_next(a, w);
+    }
+  }
+
+  // ---- teardown: every thread arrives here, on success and on abort ----
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    __syncwarp();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kCols) : "memory");
+  }
+}
+
+bool plan_t_layout(int np, int rows_box, TLayout* lay) {
+  lay->rows_box = rows_box;
+  lay->q_half = np * 128;
+  lay->q_bytes = 2 * lay->q_half;
+  const int fixed = 2 * lay->q_bytes + 2 * kPBytes + kMiscBytes;
+  int n_kv = (227 * 1024 - fixed) / kKvBytes;
+  if (n_kv > kTMaxKv) n_kv = kTMaxKv;
+  if (n_kv < 3) return false;
+  lay->n_kv = n_kv;
+  lay->off_q = 0;
+  lay->off_p = 2 * lay->q_bytes;
+  lay->off_kv = lay->off_p + 2 * kPBytes;
+  lay->off_misc = lay->off_kv + n_kv * kKvBytes;
+  lay->total = lay->off_misc + kMiscBytes;
+  return true;
+}
+
+template <int NP>
+int32_t launch_t(const AttnArgs& a, cudaStream_t st, int rows_pad, int grid, const TLayout& lay,
+                 const CUtensorMap& mk, const CUtensorMap& mv, const CUtensorMap& mks, const CUtensorMap& mvs,
+                 const CUtensorMap& mq) {
+  static bool configured[64] = {false};
+  int dev = 0;
+  MS_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev >= 0 && dev < 64 && !configured[dev]) {
+    MS_CUDA_TRY(cudaFuncSetAttribute(attn_umma_t_kernel<NP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     227 * 1024));
+    configured[dev] = true;
+  }
+  if (a.ev_split_begin) MS_CUDA_TRY(cudaEventRecord(a.ev_split_begin, st));
+  attn_umma_t_kernel<NP><<<grid, kTThreads, lay.total, st>>>(a, mk, mv, mks, mvs, mq, rows_pad, lay);
+  MS_LAUNCH_CHECK();
+  if (a.ev_split_end) MS_CUDA_TRY(cudaEventRecord(a.ev_split_end, st));
+  return MS_OK;
+}
+
+}  // namespace
+
+bool attn_umma_t_supports(int D, int G, int max_nq) { return D == 128 && G * max_nq <= 64; }
+
+int32_t launch_attn_umma_t(const AttnArgs& a, cudaStream_t st) {
+  if (a.B == 0 || a.T == 0) return MS_OK;
+  const int rows = a.max_nq * a.G;
+  const int rows_pad = (rows + 15) & ~15;
+  TLayout lay;
+  if (!attn_umma_t_supports(a.D, a.G, a.max_nq) || !plan_t_layout(rows_pad, rows, &lay))
+    return MS_ERR_UNSUPPORTED_SHAPE;
+  if (static_cast<int>((a.B + 1 + kTThreads) * sizeof(int)) > lay.off_misc) return MS_ERR_UNSUPPORTED_SHAPE;
+  const int grid = attn_mma_grid();
+  if (grid <= 0) return cuda_status(cudaErrorNoDevice);
+  CUtensorMap mk, mv, mks, mvs, mq;
+  const bool ok =
+      make_map(&mk, a.k_cache, a.D, static_cast<uint64_t>(a.n_slots), a.H_kv, a.D, a.kv_head_stride, kTile, 1) &&
+      make_map(&mv, a.v_cache, a.D, static_cast<uint64_t>(a.n_slots), a.H_kv, a.D, a.kv_head_stride, kTile, 1) &&
+      make_map(&mks, a.k_step, a.D, a.H_kv, a.T, a.D, static_cast<uint64_t>(a.H_kv) * a.D, 1, kMaxNq) &&
+      make_map(&mvs, a.v_step, a.D, a.H_kv, a.T, a.D, static_cast<uint64_t>(a.H_kv) * a.D, 1, kMaxNq) &&
+      make_map(&mq, a.q, a.D, a.H_q, a.T, a.D, static_cast<uint64_t>(a.H_q) * a.D, a.G, a.max_nq);
+  if (!ok) return cuda_status(cudaErrorInvalidValue);
+  int32_t rc;
+  switch (rows_pad) {
+    case 16: rc = launch_t<16>(a, st, rows_pad, grid, lay, mk, mv, mks, mvs, mq); break;
+    case 32: rc = launch_t<32>(a, st, rows_pad, grid, lay, mk, mv, mks, mvs, mq); break;
+    case 48: rc = launch_t<48>(a, st, rows_pad, grid, lay, mk, mv, mks, mvs, mq); break;
+    default: rc = launch_t<64>(a, st, rows_pad, grid, lay, mk, mv, mks, mvs, mq); break;
+  }
+  if (rc != MS_OK) return rc;
+  return launch_attn_merge(a, st, rows_pad, grid);
+}
+
+}  // namespace ms
