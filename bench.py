@@ -392,11 +392,11 @@ def main():
     achieved = algo_per_launch / (split_avg_ms * 1e-3) / 1e9
     peak, peak_kind = peak_hbm()
     rows = nq * (Hq // Hkv)
-    use_umma = args.attn_path == "tcgen05" or (args.attn_path == "auto" and rows > 32)
-    if args.attn_path == "tcgen05_keys":
-        kernel_name = f"attn_umma_t_kernel<{(rows + 15) // 16 * 16}>"
-    else:
-        kernel_name = "attn_umma_kernel<128>" if use_umma else f"attn_split_kernel<128,{1 if rows <= 16 else 2 if rows <= 32 else 4}>"
+    path = args.attn_path
+    if path == "auto":
+        path = "tcgen05_keys" if rows <= 64 else "tcgen05"
+    kernel_name = {"tcgen05_keys": f"attn_umma_t_kernel<{(rows + 15) // 16 * 16}>", "tcgen05": "attn_umma_kernel<128>",
+                   "mma_sync": f"attn_split_kernel<128,{1 if rows <= 16 else 2 if rows <= 32 else 4}>"}[path]
     roofline = {"bound": "hbm", "kernel": kernel_name, "achieved": achieved, "peak": peak,
                 "peak_source": f"{peak_kind} copy bandwidth", "unit": "GB/s", "frac": achieved / peak,
                 "frac_of_nominal_8000": achieved / 8000.0, "avg_launch_ms": split_avg_ms,

@@ -156,18 +156,20 @@ MS_API size_t memosight_attn_workspace_bytes(int32_t batch, int32_t n_q_heads, i
 /* Queues the attention of one layer (split-KV pass + log-sum-exp merge).
  * Limits: n_q_heads/n_kv_heads <= 16; max_nq <= 16; batch <= 8192 per call.
  * Blocks with max_nq * (H_q/H_kv) <= 128 and D in {64,128} take a tensor-core
- * path (mma.sync up to 32 packed rows, tcgen05 above); anything else inside the
- * limits takes the slower general path.
+ * path (see memosight_attn_set_path); anything else inside the limits takes the
+ * slower general path.
  * The workspace may be reused by the next call on the same stream; two calls
  * that overlap on the GPU need two workspaces. */
 MS_API int32_t memosight_attn_step(const memosight_attn_params* params, memosight_stream_t stream);
 
 /* Diagnostic switch: which kernel memosight_attn_step uses from now on, process-wide.
- * MS_ATTN_PATH_AUTO (the default) picks by shape: the mma.sync kernel up to 32 packed rows
- * (max_nq * H_q/H_kv), the tcgen05 kernel up to 128, the general kernel otherwise.  Forcing a
- * path that does not cover a shape falls back to the automatic choice for that call.  Returns
- * the previous setting, or MS_ERR_INVALID_ARG.  Results of all paths agree within the
- * tolerance of bf16 inputs with fp32 accumulation; the switch exists for tests and timing. */
+ * MS_ATTN_PATH_AUTO (the default) picks by shape: head_dim 128 with up to 64 packed rows
+ * (max_nq * H_q/H_kv) takes the keys-on-lanes tcgen05 kernel, 65..128 rows the rows-on-lanes
+ * tcgen05 kernel, head_dim 64 the mma.sync kernel (up to 64 rows), anything else the general
+ * kernel.  Forcing a path that does not cover a shape falls back to the automatic choice for
+ * that call.  Returns the previous setting, or MS_ERR_INVALID_ARG.  Results of all paths agree
+ * within the tolerance of bf16 inputs with fp32 accumulation; the switch exists for tests and
+ * timing. */
 #define MS_ATTN_PATH_AUTO 0
 #define MS_ATTN_PATH_MMA_SYNC 1
 #define MS_ATTN_PATH_TCGEN05 2

@@ -17,9 +17,10 @@ bool fast_path_shape(int D, int G, int max_nq) {
   return mma_shape(D, G, max_nq) || ms::attn_umma_supports(D, G, max_nq);
 }
 
-// Which kernel serves a shape: blocks of up to 32 packed rows stream fastest through the
-// mma.sync kernel; above that every K/V byte would be re-read from shared memory once per
-// 16-row block, so the tcgen05 kernel (operands straight from shared memory) takes over.
+// Which kernel serves a shape.  head_dim 128 with up to 64 packed rows -- every step block of
+// the method -- streams fastest through the keys-on-lanes tcgen05 kernel, whose softmax cost
+// follows the block size; 65..128 rows take the rows-on-lanes tcgen05 kernel; head_dim 64
+// stays on the mma.sync kernel up to 64 rows.
 int32_t pick_path(int D, int G, int max_nq) {
   const int32_t forced = g_forced_path.load(std::memory_order_relaxed);
   const bool mma_ok = mma_shape(D, G, max_nq), umma_ok = ms::attn_umma_supports(D, G, max_nq);
@@ -28,7 +29,8 @@ int32_t pick_path(int D, int G, int max_nq) {
   if (forced == MS_ATTN_PATH_TCGEN05 && umma_ok) return forced;
   if (forced == MS_ATTN_PATH_TCGEN05_KEYS && umma_t_ok) return forced;
   if (forced == MS_ATTN_PATH_GENERAL) return forced;
-  if (mma_ok && (max_nq * G <= 32 || !umma_ok)) return MS_ATTN_PATH_MMA_SYNC;
+  if (umma_t_ok) return MS_ATTN_PATH_TCGEN05_KEYS;
+  if (mma_ok) return MS_ATTN_PATH_MMA_SYNC;
   if (umma_ok) return MS_ATTN_PATH_TCGEN05;
   return MS_ATTN_PATH_GENERAL;
 }

@@ -30,7 +30,7 @@
 namespace ms {
 namespace {
 
-constexpr int kTThreads = 256;
+constexpr int kTThreads = 384;   // warp 0: TMA, warp 1: MMA issue, 4-7 and 8-11: the two softmax warpgroups
 constexpr float kGrowLimit = 48.f;
 constexpr int kTMaxKv = 8;
 constexpr int kPBytes = kTile * 128;            // P^T tile: 128 keys x 64 columns of bf16
@@ -40,9 +40,9 @@ constexpr uint32_t kHalfStrideT = kTile * 128;  // bytes between the 64-column h
 enum : int {
   kTbKvFull = 0, kTbKvEmpty = kTMaxKv, kTbQFull = 2 * kTMaxKv, kTbQEmpty = kTbQFull + 2,
   kTbSFull = kTbQEmpty + 2, kTbPFull = kTbSFull + 2, kTbPvDone = kTbPFull + 2, kTbWg = kTbPvDone + 2,
-  kTbDrain = kTbWg + 1, kTbCount = kTbDrain + 1
+  kTbDrain = kTbWg + 2, kTbCount = kTbDrain + 1
 };
-// misc region behind the ring: barriers | scalars | m_ref[64] | red[4][64]
+// misc region behind the ring: barriers | scalars | m_ref[64] | red[2 warpgroups][4 warps][32 rows]
 constexpr int kMiscScalars = 256, kMiscMref = 512, kMiscRed = 768, kMiscBytes = 2048;
 static_assert(kTbCount * 8 <= kMiscScalars, "barriers overflow their slot");
 
@@ -74,7 +74,7 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
                    const __grid_constant__ CUtensorMap map_vs, const __grid_constant__ CUtensorMap map_q,
                    int rows_pad, const TLayout lay) {
   constexpr int D = 128, HALVES = 2, KSTEPS_QK = D / 16;
-  constexpr int GROUPS = (NP + 31) / 32;
+  constexpr int CW = NP / 2;                        // rows (score columns) per softmax warpgroup
   constexpr uint32_t kCols = NP <= 16 ? 64 : (NP <= 32 ? 128 : 256);   // S^T x2 and O^T, a power of two
   constexpr uint32_t kColO = 2 * NP;
   extern __shared__ __align__(1024) uint8_t smem[];
@@ -82,7 +82,7 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
   const uint32_t bars = sb + lay.off_misc;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + lay.off_misc + kMiscScalars);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + lay.off_misc + kMiscScalars + 8);
-  volatile int* grow_flag = reinterpret_cast<volatile int*>(smem + lay.off_misc + kMiscScalars + 16);
+  volatile int* grow_flags = reinterpret_cast<volatile int*>(smem + lay.off_misc + kMiscScalars + 16);
   float* s_mref = reinterpret_cast<float*>(smem + lay.off_misc + kMiscMref);
   float* s_red = reinterpret_cast<float*>(smem + lay.off_misc + kMiscRed);
   uint32_t* status = reinterpret_cast<uint32_t*>(a.workspace);
@@ -125,13 +125,15 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
       mbar_init(bars + 8 * (kTbQFull + i), 1);
       mbar_init(bars + 8 * (kTbQEmpty + i), 1);
       mbar_init(bars + 8 * (kTbSFull + i), 1);
-      mbar_init(bars + 8 * (kTbPFull + i), 4);
+      mbar_init(bars + 8 * (kTbPFull + i), 8);
       mbar_init(bars + 8 * (kTbPvDone + i), 1);
     }
     mbar_init(bars + 8 * kTbWg, 4);
+    mbar_init(bars + 8 * (kTbWg + 1), 4);
     mbar_init(bars + 8 * kTbDrain, 1);
     *abort_flag = 0;
-    *grow_flag = 0;
+    grow_flags[0] = 0;
+    grow_flags[1] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();   // the prefix has been consumed
@@ -164,6 +166,8 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
     Walk w = w0;
     bool ok = true;
     int uses = 0, pieces = 0;
+    RingPos rp;
+    rp.init(0, lay.n_kv);
     while (w.it < n_iter) {
       walk_tile(a, w);
       if (w.first) {
@@ -183,12 +187,12 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
       }
 #pragma unroll 1
       for (int kv = 0; kv < 2; ++kv) {
-        const int use = 2 * w.it + kv;
-        const int buf = use % lay.n_kv;
-        if (!mbar_wait(bars + 8 * (kTbKvEmpty + buf), ((use / lay.n_kv) & 1) ^ 1, abort_flag, status)) {
+        const int buf = rp.buf;
+        if (!mbar_wait(bars + 8 * (kTbKvEmpty + buf), rp.par ^ 1u, abort_flag, status)) {
           ok = false;
           break;
         }
+        rp.step(1);
         fence_async_smem();
         const uint32_t dst = sb + lay.off_kv + buf * kKvBytes;
         const uint32_t bar = bars + 8 * (kTbKvFull + buf);
@@ -216,82 +220,102 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
       (void)mbar_wait(bars + 8 * (kTbQFull + (p & 1)), (p >> 1) & 1, abort_flag, status);
   } else if (warp == 1 && lane == 0 && n_iter > 0) {
     // =========================== MMA issuer ===========================
-    const uint32_t idesc_qk = instr_desc(NP, 0, 0);     // A = K tile (K-major), B = Q (K-major)
-    const uint32_t idesc_pv = instr_desc(NP, 1, 1);     // A = V tile^T (MN-major), B = P^T (MN-major)
+    // S^T = K Q^T: A = K tile (K-major), B = Q (K-major).  O^T += V^T P^T: A = V tile transposed
+    // (MN-major), B = P^T (MN-major).  Q K^T runs one tile ahead of the PV product, so the tensor
+    // pipe has the scores of tile t+1 ready while the softmax of tile t is in flight.  The
+    // descriptors differ from MMA to MMA only by a constant in their low word.
+    const uint32_t idesc_qk = instr_desc(NP, 0, 0), idesc_pv = instr_desc(NP, 1, 1);
+    const uint32_t q_lo0 = desc_lo(sb + lay.off_q, 16), k_lo0 = desc_lo(sb + lay.off_kv, 16);
+    const uint32_t p_lo0 = desc_lo(sb + lay.off_p, kHalfStrideT), v_lo0 = desc_lo(sb + lay.off_kv, kHalfStrideT);
     Walk wq = w0, wp = w0;
+    RingPos rk, rv;
+    rk.init(0, lay.n_kv);
+    rv.init(1, lay.n_kv);
     bool ok = true;
     auto issue_qk = [&]() -> bool {
       walk_tile(a, wq);
       const int it = wq.it, qb = wq.piece_idx & 1;
-      if (wq.first &&
-          !mbar_wait(bars + 8 * (kTbQFull + qb), (wq.piece_idx >> 1) & 1, abort_flag, status))
+      if ((wq.first && !mbar_wait(bars + 8 * (kTbQFull + qb), (wq.piece_idx >> 1) & 1, abort_flag, status)) ||
+          !mbar_wait(bars + 8 * (kTbKvFull + rk.buf), rk.par, abort_flag, status))
         return false;
-      const int use = 2 * it, buf = use % lay.n_kv;
-      if (!mbar_wait(bars + 8 * (kTbKvFull + buf), (use / lay.n_kv) & 1, abort_flag, status)) return false;
       tc_fence_after();
-      const uint32_t qa = sb + lay.off_q + qb * lay.q_bytes;
-      const uint32_t ka = sb + lay.off_kv + buf * kKvBytes;
+      const uint32_t q_lo = q_lo0 + qb * (lay.q_bytes >> 4);
+      const uint32_t k_lo = k_lo0 + rk.buf * (kKvBytes >> 4);
       const uint32_t d_s = tmem + (it & 1) * NP;
 #pragma unroll
-      for (int ks = 0; ks < KSTEPS_QK; ++ks) {
-        const uint32_t koff = (ks >> 2) * kHalfStrideT + (ks & 3) * 32;
-        const uint32_t qoff = (ks >> 2) * lay.q_half + (ks & 3) * 32;
-        umma_bf16(d_s, smem_desc(ka + koff, 16), smem_desc(qa + qoff, 16), idesc_qk, ks > 0);
-      }
-      umma_commit(bars + 8 * (kTbKvEmpty + buf));
+      for (int ks = 0; ks < KSTEPS_QK; ++ks)
+        umma_bf16_lo(d_s, k_lo + (ks >> 2) * (kHalfStrideT >> 4) + (ks & 3) * 2,
+                     q_lo + (ks >> 2) * (NP * 128 >> 4) + (ks & 3) * 2, idesc_qk, ks > 0);
+      umma_commit(bars + 8 * (kTbKvEmpty + rk.buf));
       umma_commit(bars + 8 * (kTbSFull + (it & 1)));
       if (wq.last) umma_commit(bars + 8 * (kTbQEmpty + qb));
+      rk.step(2);
       walk_next(a, wq);
       return true;
     };
     ok = issue_qk();
     while (ok && wp.it < n_iter) {
+      // score buffer (it+1)&1 is free: the P^T of tile it-1 was waited for in the previous round
       if (wq.it < n_iter && !issue_qk()) { ok = false; break; }
       walk_tile(a, wp);
       const int it = wp.it;
-      const int use = 2 * it + 1, buf = use % lay.n_kv;
       if (!mbar_wait(bars + 8 * (kTbPFull + (it & 1)), (it >> 1) & 1, abort_flag, status) ||
-          !mbar_wait(bars + 8 * (kTbKvFull + buf), (use / lay.n_kv) & 1, abort_flag, status)) {
+          !mbar_wait(bars + 8 * (kTbKvFull + rv.buf), rv.par, abort_flag, status)) {
         ok = false;
         break;
       }
       tc_fence_after();
-      const uint32_t pa = sb + lay.off_p + (it & 1) * kPBytes;
-      const uint32_t va = sb + lay.off_kv + buf * kKvBytes;
+      const uint32_t p_lo = p_lo0 + (it & 1) * (kPBytes >> 4);
+      const uint32_t v_lo = v_lo0 + rv.buf * (kKvBytes >> 4);
       const int ksteps = wp.is_step ? 1 : (wp.nvalid + 15) >> 4;
+      const uint32_t acc0 = wp.first ? 0u : 1u;
+      if (ksteps == kTile / 16) {
+#pragma unroll
+        for (int j = 0; j < kTile / 16; ++j)
+          umma_bf16_lo(tmem + kColO, v_lo + j * (2048 >> 4), p_lo + j * (2048 >> 4), idesc_pv, j == 0 ? acc0 : 1u);
+      } else {
 #pragma unroll 1
-      for (int j = 0; j < ksteps; ++j)
-        umma_bf16(tmem + kColO, smem_desc(va + j * 2048, kHalfStrideT), smem_desc(pa + j * 2048, kHalfStrideT),
-                  idesc_pv, !(wp.first && j == 0));
-      umma_commit(bars + 8 * (kTbKvEmpty + buf));
+        for (int j = 0; j < ksteps; ++j)
+          umma_bf16_lo(tmem + kColO, v_lo + j * (2048 >> 4), p_lo + j * (2048 >> 4), idesc_pv, j == 0 ? acc0 : 1u);
+      }
+      umma_commit(bars + 8 * (kTbKvEmpty + rv.buf));
       umma_commit(bars + 8 * (kTbPvDone + (it & 1)));
+      rv.step(2);
       walk_next(a, wp);
     }
     if (!ok) {
+      // aborting: let the tensor pipe run dry before tensor memory is released
       umma_commit(bars + 8 * kTbDrain);
       const unsigned long long t_begin = global_ns();
       while (!mbar_try_wait(bars + 8 * kTbDrain, 0) && global_ns() - t_begin < kWaitLimitNs) {
       }
     }
   } else if (warp >= 4 && n_iter > 0) {
-    // =========================== softmax warps: thread = key of the tile ===========================
-    const int quad = warp - 4;
+    // ============ softmax warps: thread = key of the tile; warpgroup = half of the rows ============
+    // Rows (score columns) are independent of one another, so the two warpgroups never talk:
+    // each has its own references, partial sums, agreement barrier and share of every P^T row.
+    const int wg = (warp - 4) >> 2, quad = (warp - 4) & 3;
     const int t = quad * 32 + lane;                        // key index in the tile = TMEM lane
+    const int c0 = wg * CW;                                // first row (score column) of this warpgroup
     const uint32_t lane_addr = tmem + (static_cast<uint32_t>(quad * 32) << 16);
     const uint32_t tx = t & 7;
-    float* red_w = s_red + quad * 64;
+    float* red_w = s_red + (wg * 4 + quad) * 32;
+    const float* red_g = s_red + wg * 128;                 // this warpgroup's four slices
+    float* mref_g = s_mref + c0;
+    volatile int* grow_flag = grow_flags + wg;
+    const uint32_t bar_wg = bars + 8 * (kTbWg + wg);
     Walk w = w0;
-    float lsum[NP];
+    float lsum[CW];
     uint32_t wg_phase = 0;
     bool ok = true;
     auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {
       return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, status));
     };
-    // bounded barrier of the four softmax warps (also publishes their shared-memory writes)
+    // bounded barrier of the warpgroup's four warps (also publishes their shared-memory writes)
     auto wg_sync = [&]() -> bool {
       __syncwarp();
-      if (lane == 0) mbar_arrive(bars + 8 * kTbWg);
-      const bool good = wait_all(bars + 8 * kTbWg, wg_phase & 1);
+      if (lane == 0) mbar_arrive(bar_wg);
+      const bool good = wait_all(bar_wg, wg_phase & 1);
       ++wg_phase;
       return good;
     };
@@ -309,30 +333,30 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
         if (!wait_all(bars + 8 * (kTbKvFull + buf), (use / lay.n_kv) & 1)) { ok = false; break; }
         const uint32_t va = sb + lay.off_kv + buf * kKvBytes;
         const int n_rows = ((nv + 15) & ~15) - nv;
-        for (int x = t; x < n_rows * HALVES * 8; x += 128) {
+        for (int x = wg * 128 + t; x < n_rows * HALVES * 8; x += 256) {
           const int rr = nv + x / (HALVES * 8), cc = x % (HALVES * 8);
           const uint32_t addr = va + (cc >> 3) * kHalfStrideT + rr * 128 + ((cc & 7) << 4);
           asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(addr), "r"(0u) : "memory");
         }
       }
       const bool key_ok = t < nv;
-      const uint32_t s_addr = lane_addr + pb * NP;
+      const uint32_t s_addr = lane_addr + pb * NP + c0;
 
-      // scores of this key against every row; invisible pairs become -inf
-      float v[NP];
+      // scores of this key against the warpgroup's rows; invisible pairs become -inf
+      float v[CW];
       auto load_scores = [&]() {
-        uint32_t raw[NP];
+        uint32_t raw[CW];
 #pragma unroll
-        for (int c = 0; c < NP / 16; ++c) tmem_ld16(s_addr + c * 16, raw + c * 16);
+        for (int c = 0; c < CW / 8; ++c) tmem_ld8(s_addr + c * 8, raw + c * 8);
 #pragma unroll
-        for (int c = 0; c < NP / 16; ++c) tmem_ld_wait16(raw + c * 16);
+        for (int c = 0; c < CW / 8; ++c) tmem_ld_wait8(raw + c * 8);
         if (!w.is_step) {
 #pragma unroll
-          for (int j = 0; j < NP; ++j) v[j] = key_ok ? __uint_as_float(raw[j]) : -INFINITY;
+          for (int j = 0; j < CW; ++j) v[j] = key_ok ? __uint_as_float(raw[j]) : -INFINITY;
         } else {
-          int i = 0, g = 0;
+          int i = c0 / a.G, g = c0 - i * a.G;
 #pragma unroll
-          for (int j = 0; j < NP; ++j) {
+          for (int j = 0; j < CW; ++j) {
             bool vis = false;
             if (key_ok && i < w.n_q) {
               const int anc = (i < w.n_c) ? i : (a.anchor ? a.anchor[w.r0 + i] : w.n_c);
@@ -345,16 +369,16 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
       };
       // exact maximum over the tile's keys of every row -> red[warp][row]
       auto reduce_row_max = [&]() {
-        float keep[GROUPS];
+        float keep = -INFINITY;
 #pragma unroll
-        for (int g = 0; g < GROUPS; ++g) keep[g] = -INFINITY;
-#pragma unroll
-        for (int j = 0; j < NP; ++j) {
+        for (int j = 0; j < CW; ++j) {
           const float r = warp_max_f32(v[j]);
-          if (lane == (j & 31)) keep[j >> 5] = r;
+          if (lane == j) keep = r;
         }
-#pragma unroll
-        for (int g = 0; g < GROUPS; ++g) red_w[g * 32 + lane] = keep[g];
+        red_w[lane] = keep;
+      };
+      auto red_max4 = [&](int j) -> float {
+        return fmaxf(fmaxf(red_g[j], red_g[32 + j]), fmaxf(red_g[64 + j], red_g[96 + j]));
       };
       load_scores();
 
@@ -362,20 +386,20 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
         // new unit: the reference maximum of each row is the exact maximum of this first tile
         reduce_row_max();
         if (!wg_sync()) { ok = false; break; }
-        if (t < NP) {
-          const float m = fmaxf(fmaxf(s_red[t], s_red[64 + t]), fmaxf(s_red[128 + t], s_red[192 + t]));
-          s_mref[t] = (m == -INFINITY) ? 0.f : m * a.scale_log2;
+        if (t < CW) {
+          const float m = red_max4(t);
+          mref_g[t] = (m == -INFINITY) ? 0.f : m * a.scale_log2;
         }
         if (!wg_sync()) { ok = false; break; }
 #pragma unroll
-        for (int j = 0; j < NP; ++j) lsum[j] = 0.f;
+        for (int j = 0; j < CW; ++j) lsum[j] = 0.f;
       }
 
       // x = s * scale - m_ref (log2 units)
       float tmaxx = -INFINITY;
 #pragma unroll
-      for (int j4 = 0; j4 < NP / 4; ++j4) {
-        const float4 m4 = *reinterpret_cast<const float4*>(s_mref + 4 * j4);
+      for (int j4 = 0; j4 < CW / 4; ++j4) {
+        const float4 m4 = *reinterpret_cast<const float4*>(mref_g + 4 * j4);
         v[4 * j4 + 0] = fmaf(v[4 * j4 + 0], a.scale_log2, -m4.x);
         v[4 * j4 + 1] = fmaf(v[4 * j4 + 1], a.scale_log2, -m4.y);
         v[4 * j4 + 2] = fmaf(v[4 * j4 + 2], a.scale_log2, -m4.z);
@@ -390,34 +414,34 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
         load_scores();
         reduce_row_max();
         if (!wg_sync()) { ok = false; break; }
-        float alpha[NP];
+        float alpha[CW];
 #pragma unroll
-        for (int j = 0; j < NP; ++j) {
-          const float m = fmaxf(fmaxf(s_red[j], s_red[64 + j]), fmaxf(s_red[128 + j], s_red[192 + j]));
-          const float m_old = s_mref[j];
+        for (int j = 0; j < CW; ++j) {
+          const float m = red_max4(j);
+          const float m_old = mref_g[j];
           const float m_new = (m == -INFINITY) ? m_old : fmaxf(m_old, m * a.scale_log2);
           alpha[j] = ex2(m_old - m_new);
           lsum[j] *= alpha[j];
           v[j] = fmaf(v[j], a.scale_log2, -m_new);
         }
         if (!wg_sync()) { ok = false; break; }          // everyone has read the old references
-        if (t < NP) {
-          const float m = fmaxf(fmaxf(s_red[t], s_red[64 + t]), fmaxf(s_red[128 + t], s_red[192 + t]));
-          if (m != -INFINITY) s_mref[t] = fmaxf(s_mref[t], m * a.scale_log2);
+        if (t < CW) {
+          const float m = red_max4(t);
+          if (m != -INFINITY) mref_g[t] = fmaxf(mref_g[t], m * a.scale_log2);
         }
         // all PV products issued so far are complete before O^T is touched
         if (!wait_all(bars + 8 * (kTbPvDone + ((it - 1) & 1)), ((it - 1) >> 1) & 1)) { ok = false; break; }
         tc_fence_after();
         {
-          uint32_t o[NP];
+          uint32_t o[CW];
 #pragma unroll
-          for (int c = 0; c < NP / 16; ++c) tmem_ld16(lane_addr + kColO + c * 16, o + c * 16);
+          for (int c = 0; c < CW / 8; ++c) tmem_ld8(lane_addr + kColO + c0 + c * 8, o + c * 8);
 #pragma unroll
-          for (int c = 0; c < NP / 16; ++c) tmem_ld_wait16(o + c * 16);
+          for (int c = 0; c < CW / 8; ++c) tmem_ld_wait8(o + c * 8);
 #pragma unroll
-          for (int j = 0; j < NP; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha[j]);
+          for (int j = 0; j < CW; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha[j]);
 #pragma unroll
-          for (int c = 0; c < NP / 16; ++c) tmem_st16(lane_addr + kColO + c * 16, o + c * 16);
+          for (int c = 0; c < CW / 8; ++c) tmem_st8(lane_addr + kColO + c0 + c * 8, o + c * 8);
           asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
         }
         if (!wg_sync()) { ok = false; break; }          // new references visible to later tiles
@@ -427,14 +451,14 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
       {
         const uint32_t p_row = sb + lay.off_p + pb * kPBytes + t * 128;
 #pragma unroll
-        for (int c = 0; c < NP / 8; ++c) {
+        for (int c = 0; c < CW / 8; ++c) {
           float p[8];
 #pragma unroll
           for (int e = 0; e < 8; ++e) {
             p[e] = ex2(v[c * 8 + e]);
             lsum[c * 8 + e] += p[e];
           }
-          const uint32_t addr = p_row + ((c ^ tx) << 4);
+          const uint32_t addr = p_row + (((c0 / 8 + c) ^ tx) << 4);
           asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(pack2(p[0], p[1])),
                        "r"(pack2(p[2], p[3])), "r"(pack2(p[4], p[5])), "r"(pack2(p[6], p[7]))
                        : "memory");
@@ -448,33 +472,32 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
       if (w.last) {
         // ---- end of the unit (or of this CTA's part of it) ----
         // row sums: over the 32 lanes of each warp, then over the four warps
-#pragma unroll
-        for (int g = 0; g < GROUPS; ++g) {
+        {
           float tsum[32];
 #pragma unroll
-          for (int i = 0; i < 32; ++i) tsum[i] = (g * 32 + i < NP) ? lsum[(g * 32 + i < NP) ? g * 32 + i : 0] : 0.f;
-          red_w[g * 32 + lane] = warp_sum_32rows(tsum, lane);
+          for (int i = 0; i < 32; ++i) tsum[i] = (i < CW) ? lsum[i < CW ? i : 0] : 0.f;
+          red_w[lane] = warp_sum_32rows(tsum, lane);
         }
         if (!wg_sync()) { ok = false; break; }
         const int rows = w.n_q * a.G;
-        float l_row[NP];
+        float l_row[CW];
 #pragma unroll
-        for (int j = 0; j < NP; ++j) l_row[j] = (s_red[j] + s_red[64 + j]) + (s_red[128 + j] + s_red[192 + j]);
-        const float m_mine = (t < NP) ? s_mref[t] : 0.f;
+        for (int j = 0; j < CW; ++j) l_row[j] = (red_g[j] + red_g[32 + j]) + (red_g[64 + j] + red_g[96 + j]);
+        const float m_mine = (t < CW) ? mref_g[t] : 0.f;
         if (!wg_sync()) { ok = false; break; }          // red and m_ref may be reused from here on
         if (!wait_all(bars + 8 * (kTbPvDone + pb), (it >> 1) & 1)) { ok = false; break; }
         tc_fence_after();
-        uint32_t o[NP];
+        uint32_t o[CW];
 #pragma unroll
-        for (int c = 0; c < NP / 16; ++c) tmem_ld16(lane_addr + kColO + c * 16, o + c * 16);
+        for (int c = 0; c < CW / 8; ++c) tmem_ld8(lane_addr + kColO + c0 + c * 8, o + c * 8);
 #pragma unroll
-        for (int c = 0; c < NP / 16; ++c) tmem_ld_wait16(o + c * 16);
+        for (int c = 0; c < CW / 8; ++c) tmem_ld_wait8(o + c * 8);
         // thread t holds element d = t of every row
         if (w.slot < 0) {
-          int i = 0, g = 0;
+          int i = c0 / a.G, g = c0 - i * a.G;
 #pragma unroll
-          for (int j = 0; j < NP; ++j) {
-            if (j < rows) {
+          for (int j = 0; j < CW; ++j) {
+            if (c0 + j < rows) {
               const int64_t orow = static_cast<int64_t>(w.r0 + i) * a.H_q + w.h * a.G + g;
               a.out[orow * D + t] = __float2bfloat16_rn(__uint_as_float(o[j]) / l_row[j]);
               if (a.lse && t == j) a.lse[orow] = (m_mine + log2f(l_row[j])) * 0.69314718055994531f;
@@ -485,12 +508,12 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
           float* slot = ws_slots + static_cast<size_t>(w.slot) * ws_slot_floats(D, rows_pad);
           float* sm = slot + static_cast<size_t>(rows_pad) * D;
 #pragma unroll
-          for (int j = 0; j < NP; ++j) {
-            if (j < rows) {
-              slot[static_cast<size_t>(j) * D + t] = __uint_as_float(o[j]);
+          for (int j = 0; j < CW; ++j) {
+            if (c0 + j < rows) {
+              slot[static_cast<size_t>(c0 + j) * D + t] = __uint_as_float(o[j]);
               if (t == j) {
-                sm[j] = m_mine;
-                sm[rows_pad + j] = l_row[j];
+                sm[c0 + j] = m_mine;
+                sm[rows_pad + c0 + j] = l_row[j];
               }
             }
           }
