@@ -43,7 +43,7 @@ UNIT = "tokens/s"
 SEG_LEN, MEM_TOKENS = 512, 170          # one compaction: 512-token step -> 170 memory tokens + <o>
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes the split kernel moved per algorithmic byte in the ncu capture summarised in
-# profiles/attn_split_kernel_sweep_b32_L16384.md (batch 32; scaled by the bytes streamed).
+# profiles/attn_umma_t_kernel_sweep_b32_L16384.md (batch 32; scaled by the bytes streamed).
 NCU_TRAFFIC_PER_ALGO_BYTE = 1.011
 KERNELS_PER_STEP = 9                    # rope 1, attention 2, accept 2, append 2, compaction 2
 
