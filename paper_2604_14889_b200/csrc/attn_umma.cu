@@ -190,6 +190,8 @@ attn_umma_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
     bool ok = true;
     int uses = 0;                      // K/V buffer fills issued
     int pieces = 0;                    // Q fills issued
+    RingPos rp;
+    rp.init(0, lay.n_kv);
     while (w.it < n_iter) {
       walk_tile(a, w);
       if (w.first) {
@@ -209,12 +211,12 @@ attn_umma_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
       }
 #pragma unroll 1
       for (int kv = 0; kv < 2; ++kv) {
-        const int use = 2 * w.it + kv;
-        const int buf = use % lay.n_kv;
-        if (!mbar_wait(bars + 8 * (kBarKvEmpty + buf), ((use / lay.n_kv) & 1) ^ 1, abort_flag, status)) {
+        const int buf = rp.buf;
+        if (!mbar_wait(bars + 8 * (kBarKvEmpty + buf), rp.par ^ 1u, abort_flag, status)) {
           ok = false;
           break;
         }
+        rp.step(1);
         fence_async_smem();
         const uint32_t dst = sb + lay.off_kv + buf * lay.kv_bytes;
         const uint32_t bar = bars + 8 * (kBarKvFull + buf);
@@ -242,32 +244,35 @@ attn_umma_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
       (void)mbar_wait(bars + 8 * (kBarQFull + (p & 1)), (p >> 1) & 1, abort_flag, status);
   } else if (warp == 1 && lane == 0 && n_iter > 0) {
     // =========================== MMA issuer ===========================
+    // The descriptors of consecutive MMAs differ only by a constant in their low word.
     const uint32_t idesc_qk = instr_desc(kTile, 0), idesc_qk_step = instr_desc(kMaxNq, 0);
     const uint32_t idesc_pv = instr_desc(D, 1);
+    const uint32_t q_lo0 = desc_lo(sb + lay.off_q, 16), k_lo0 = desc_lo(sb + lay.off_kv, 16);
+    const uint32_t p_lo0 = desc_lo(sb + lay.off_p, 16), v_lo0 = desc_lo(sb + lay.off_kv, kHalfStride);
     Walk wq = w0, wp = w0;
+    RingPos rk, rv;
+    rk.init(0, lay.n_kv);
+    rv.init(1, lay.n_kv);
     bool ok = true;
     auto issue_qk = [&]() -> bool {
       walk_tile(a, wq);
       const int it = wq.it, qb = wq.piece_idx & 1;
-      if (wq.first &&
-          !mbar_wait(bars + 8 * (kBarQFull + qb), (wq.piece_idx >> 1) & 1, abort_flag, status))
+      if ((wq.first && !mbar_wait(bars + 8 * (kBarQFull + qb), (wq.piece_idx >> 1) & 1, abort_flag, status)) ||
+          !mbar_wait(bars + 8 * (kBarKvFull + rk.buf), rk.par, abort_flag, status))
         return false;
-      const int use = 2 * it, buf = use % lay.n_kv;
-      if (!mbar_wait(bars + 8 * (kBarKvFull + buf), (use / lay.n_kv) & 1, abort_flag, status)) return false;
       tc_fence_after();
-      const uint32_t qa = sb + lay.off_q + qb * lay.q_bytes;
-      const uint32_t ka = sb + lay.off_kv + buf * lay.kv_bytes;
+      const uint32_t q_lo = q_lo0 + qb * (lay.q_bytes >> 4), q_half = lay.q_half >> 4;
+      const uint32_t k_lo = k_lo0 + rk.buf * (lay.kv_bytes >> 4);
       const uint32_t d_s = tmem + kColS + (it & 1) * kTile;
       const uint32_t idesc = wq.is_step ? idesc_qk_step : idesc_qk;
 #pragma unroll
-      for (int ks = 0; ks < KSTEPS_QK; ++ks) {
-        const uint32_t qoff = (ks >> 2) * lay.q_half + (ks & 3) * 32;
-        const uint32_t koff = (ks >> 2) * kHalfStride + (ks & 3) * 32;
-        umma_bf16(d_s, smem_desc(qa + qoff, 16), smem_desc(ka + koff, 16), idesc, ks > 0);
-      }
-      umma_commit(bars + 8 * (kBarKvEmpty + buf));
+      for (int ks = 0; ks < KSTEPS_QK; ++ks)
+        umma_bf16_lo(d_s, q_lo + (ks >> 2) * q_half + (ks & 3) * 2,
+                     k_lo + (ks >> 2) * (kHalfStride >> 4) + (ks & 3) * 2, idesc, ks > 0);
+      umma_commit(bars + 8 * (kBarKvEmpty + rk.buf));
       umma_commit(bars + 8 * (kBarSFull + (it & 1)));
       if (wq.last) umma_commit(bars + 8 * (kBarQEmpty + qb));
+      rk.step(2);
       walk_next(a, wq);
       return true;
     };
@@ -276,24 +281,30 @@ attn_umma_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
       if (wq.it < n_iter && !issue_qk()) { ok = false; break; }
       walk_tile(a, wp);
       const int it = wp.it;
-      const int use = 2 * it + 1, buf = use % lay.n_kv;
       if (!mbar_wait(bars + 8 * (kBarPFull + (it & 1)), (it >> 1) & 1, abort_flag, status) ||
-          !mbar_wait(bars + 8 * (kBarKvFull + buf), (use / lay.n_kv) & 1, abort_flag, status)) {
+          !mbar_wait(bars + 8 * (kBarKvFull + rv.buf), rv.par, abort_flag, status)) {
         ok = false;
         break;
       }
       tc_fence_after();
-      const uint32_t pa = sb + lay.off_p + (it & 1) * lay.p_bytes;
-      const uint32_t va = sb + lay.off_kv + buf * lay.kv_bytes;
+      const uint32_t p_lo = p_lo0 + (it & 1) * (lay.p_bytes >> 4), p_half = lay.p_half >> 4;
+      const uint32_t v_lo = v_lo0 + rv.buf * (lay.kv_bytes >> 4);
       const int ksteps = wp.is_step ? 1 : (wp.nvalid + 15) >> 4;
+      const uint32_t acc0 = wp.first ? 0u : 1u;
+      if (ksteps == kTile / 16) {
+#pragma unroll
+        for (int j = 0; j < kTile / 16; ++j)
+          umma_bf16_lo(tmem + kColO, p_lo + (j >> 2) * p_half + (j & 3) * 2, v_lo + j * (2048 >> 4), idesc_pv,
+                       j == 0 ? acc0 : 1u);
+      } else {
 #pragma unroll 1
-      for (int j = 0; j < ksteps; ++j) {
-        const uint32_t poff = (j >> 2) * lay.p_half + (j & 3) * 32;
-        umma_bf16(tmem + kColO, smem_desc(pa + poff, 16), smem_desc(va + j * 2048, kHalfStride), idesc_pv,
-                  !(wp.first && j == 0));
+        for (int j = 0; j < ksteps; ++j)
+          umma_bf16_lo(tmem + kColO, p_lo + (j >> 2) * p_half + (j & 3) * 2, v_lo + j * (2048 >> 4), idesc_pv,
+                       j == 0 ? acc0 : 1u);
       }
-      umma_commit(bars + 8 * (kBarKvEmpty + buf));
+      umma_commit(bars + 8 * (kBarKvEmpty + rv.buf));
       umma_commit(bars + 8 * (kBarPvDone + (it & 1)));
+      rv.step(2);
       walk_next(a, wp);
     }
     if (!ok) {
