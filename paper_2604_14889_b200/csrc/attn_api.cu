@@ -9,8 +9,11 @@
 namespace {
 
 std::atomic<int32_t> g_forced_path{MS_ATTN_PATH_AUTO};
+constexpr int32_t kPathBig = 100;   // large-block tcgen05 kernel (chosen by shape only)
 
-bool mma_shape(int D, int G, int max_nq) { return (D == 64 || D == 128) && max_nq * G <= 64; }
+bool mma_shape(int D, int G, int max_nq) {
+  return (D == 64 || D == 128) && max_nq <= ms::kMaxNq && max_nq * G <= 64;
+}
 
 // Either tensor-core path: both use the per-CTA partial slots of the split-KV workspace.
 bool fast_path_shape(int D, int G, int max_nq) {
@@ -29,6 +32,7 @@ int32_t pick_path(int D, int G, int max_nq) {
   if (forced == MS_ATTN_PATH_TCGEN05 && umma_ok) return forced;
   if (forced == MS_ATTN_PATH_TCGEN05_KEYS && umma_t_ok) return forced;
   if (forced == MS_ATTN_PATH_GENERAL) return forced;
+  if (ms::attn_umma_big_supports(D, G, max_nq)) return kPathBig;
   if (umma_t_ok) return MS_ATTN_PATH_TCGEN05_KEYS;
   if (mma_ok) return MS_ATTN_PATH_MMA_SYNC;
   if (umma_ok) return MS_ATTN_PATH_TCGEN05;
@@ -46,12 +50,13 @@ extern "C" size_t memosight_attn_workspace_bytes(int32_t batch, int32_t n_q_head
                                                  int32_t n_kv_heads, int32_t head_dim,
                                                  int32_t max_kv_len, int32_t max_nq) {
   if (batch < 0 || n_kv_heads < 1 || n_q_heads < 1 || n_q_heads % n_kv_heads || head_dim < 1 ||
-      max_kv_len < 0 || max_nq < 1 || max_nq > ms::kMaxNq)
+      max_kv_len < 0 || max_nq < 1 || max_nq > ms::kMaxNqBig)
     return 0;
   const int G = n_q_heads / n_kv_heads;
-  if (!fast_path_shape(head_dim, G, max_nq)) return ms::kWsHeaderBytes;
   int n_ctas = ms::attn_mma_grid();
   if (n_ctas <= 0) n_ctas = 256;   // no device visible: answer for the largest part we target
+  if (ms::attn_umma_big_supports(head_dim, G, max_nq)) return ms::attn_umma_big_workspace_bytes(n_ctas);
+  if (!fast_path_shape(head_dim, G, max_nq)) return ms::kWsHeaderBytes;
   const int rows_pad = (max_nq * G + 15) & ~15;
   return ms::attn_mma_workspace_bytes(head_dim, rows_pad, n_ctas);
 }
@@ -63,7 +68,7 @@ extern "C" int32_t memosight_attn_step(const memosight_attn_params* p, memosight
     return MS_ERR_INVALID_ARG;
   if (p->n_q_heads % p->n_kv_heads) return MS_ERR_INVALID_ARG;
   const int G = p->n_q_heads / p->n_kv_heads;
-  if (G > ms::kMaxGroup || p->max_nq < 1 || p->max_nq > ms::kMaxNq || p->batch > ms::kMaxBatch ||
+  if (G > ms::kMaxGroup || p->max_nq < 1 || p->max_nq > ms::kMaxNqBig || p->batch > ms::kMaxBatch ||
       p->head_dim % 32 || p->head_dim > 256 || p->n_slots >= (1ll << 31))
     return MS_ERR_UNSUPPORTED_SHAPE;
   if (p->batch == 0 || p->total_rows == 0) return MS_OK;
@@ -111,6 +116,7 @@ extern "C" int32_t memosight_attn_step(const memosight_attn_params* p, memosight
   if (path == MS_ATTN_PATH_MMA_SYNC) return ms::launch_attn_mma(a, st);
   if (path == MS_ATTN_PATH_TCGEN05) return ms::launch_attn_umma(a, st);
   if (path == MS_ATTN_PATH_TCGEN05_KEYS) return ms::launch_attn_umma_t(a, st);
+  if (path == kPathBig) return ms::launch_attn_umma_big(a, st);
   return ms::launch_attn_simt(a, st);
 }
 

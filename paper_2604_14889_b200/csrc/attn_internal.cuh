@@ -51,4 +51,10 @@ int32_t launch_attn_umma(const AttnArgs& a, cudaStream_t st);
 bool attn_umma_t_supports(int D, int G, int max_nq);
 int32_t launch_attn_umma_t(const AttnArgs& a, cudaStream_t st);
 
+// tcgen05 path for large blocks (17..256 tokens per block, head_dim 128): the block is cut
+// into row tiles; own schedule, workspace size and merge kernel.
+bool attn_umma_big_supports(int D, int G, int max_nq);
+size_t attn_umma_big_workspace_bytes(int n_ctas);
+int32_t launch_attn_umma_big(const AttnArgs& a, cudaStream_t st);
+
 }  // namespace ms

@@ -541,7 +541,7 @@ int32_t launch_umma(const AttnArgs& a, cudaStream_t st, int rows_pad, int grid, 
 
 bool attn_umma_supports(int D, int G, int max_nq) {
   UmmaLayout lay;
-  return (D == 64 || D == 128) && G * max_nq <= 128 && plan_layout(D, G * max_nq, G * max_nq, &lay);
+  return (D == 64 || D == 128) && max_nq <= kMaxNq && G * max_nq <= 128 && plan_layout(D, G * max_nq, G * max_nq, &lay);
 }
 
 int32_t launch_attn_umma(const AttnArgs& a, cudaStream_t st) {

@@ -1,0 +1,672 @@
+// tcgen05 attention for large blocks (17..256 new tokens per sequence), head_dim 128.
+//
+// MemoSight's compression pass (paper Sec. 2.1.2; Algorithm 1, the forward over the l memory
+// tokens and <o> appended behind a finished reasoning step) is the same masked attention as
+// a Predict+Verify step -- whole compacted cache visible, the block's own tokens causal -- but
+// with up to ceil(512/3)+1 = 172 tokens in the block, i.e. several hundred packed rows per KV
+// head.  The block is cut into row tiles of floor(128/G) tokens (<= 128 packed rows); a work
+// unit is (sequence, KV head, row tile) and streams the whole cache plus the step-local key
+// tiles up to its own last token (later keys are invisible to all of its rows).
+//
+// Rows on the TMEM lanes: S = Q K^T (128 x 128 per tile) and O += P V on tcgen05.mma, operands
+// from 128-byte-swizzled shared memory filled by TMA, P written by the softmax threads as the
+// K-major A operand.  The softmax is the limit in this compute-heavy regime, so two warpgroups
+// share every tile: warpgroup g takes key columns [64g, 64g+64) of the scores and, for rescales
+// and the epilogue, output columns [64g, 64g+64) of its rows.  A row's reference maximum is the
+// exact maximum of the unit's first tile (both halves, exchanged through shared memory) and only
+// moves when a score exceeds it by 2^48; the eight softmax warps agree on that through one
+// bounded mbarrier round per tile.  Row sums are kept per thread and added up at the unit's end.
+// Schedule: the flat list of all tiles of all units, cut into one contiguous range per
+// persistent CTA; a unit cut across CTAs leaves (m, l, O) partials that attn_big_merge_kernel
+// combines.  Every wait is bounded (status word in the workspace, as in the other paths).
+#include "attn_umma_common.cuh"
+
+namespace ms {
+namespace {
+
+constexpr int kBThreads = 384;    // warp 0: TMA, warp 1: MMA issue, 4-7 and 8-11: softmax warpgroups
+constexpr int kBD = 128;
+constexpr uint32_t kBCols = 512;  // S0 | S1 | O
+constexpr uint32_t kBColS = 0, kBColO = 256;
+constexpr float kBGrowLimit = 48.f;
+constexpr int kBKv = 4;                           // K/V buffers in the ring
+constexpr int kBKvBytes = kTile * kBD * 2;        // 32 KB
+constexpr uint32_t kBHalf = kTile * 128;          // bytes between 64-column halves of a tile
+constexpr int kBQBytes = 2 * kBHalf, kBPBytes = 2 * kBHalf;
+constexpr int kBOffQ = 0, kBOffP = kBQBytes, kBOffKv = kBOffP + 2 * kBPBytes;
+constexpr int kBOffMisc = kBOffKv + kBKv * kBKvBytes;
+// misc: barriers | scalars | mx[2][128] | lpart[2][128]
+constexpr int kBMiscScalars = 256, kBMiscMx = 512, kBMiscL = 1536, kBMiscBytes = 2560;
+constexpr int kBSmem = kBOffMisc + kBMiscBytes;
+static_assert(kBSmem <= 227 * 1024, "shared memory budget");
+
+enum : int {
+  kBbKvFull = 0, kBbKvEmpty = kBKv, kBbQFull = 2 * kBKv, kBbQEmpty, kBbSFull, kBbPFull = kBbSFull + 2,
+  kBbPvDone = kBbPFull + 2, kBbAll = kBbPvDone + 2, kBbDrain, kBbCount
+};
+static_assert(kBbCount * 8 <= kBMiscScalars, "barriers overflow their slot");
+
+// ---------------------------------------------------------------- schedule
+
+struct BigSeq {
+  int L, n_q, r0, n_c, cache_tiles, n_rt, tph;   // tph: tiles of one KV head (all row tiles)
+  long long slot_off;
+};
+__device__ __forceinline__ int big_step_tiles(const BigSeq& s, int rt, int tpt) {
+  const int last = min(s.n_q, (rt + 1) * tpt);           // keys up to the tile's last token
+  return (last + kTile - 1) / kTile;
+}
+__device__ __forceinline__ void big_seq(const AttnArgs& a, int b, int tpt, BigSeq& s) {
+  seq_shape(a, b, s.L, s.n_q, s.r0);
+  int n_c = a.n_cand[b];
+  s.n_c = n_c < 0 ? 0 : (n_c > s.n_q ? s.n_q : n_c);
+  s.slot_off = a.kv_off[b];
+  s.cache_tiles = (s.L + kTile - 1) / kTile;
+  s.n_rt = (s.n_q + tpt - 1) / tpt;
+  int t = s.n_rt * s.cache_tiles;
+  for (int rt = 0; rt < s.n_rt; ++rt) t += big_step_tiles(s, rt, tpt);
+  s.tph = t;
+}
+// Exclusive prefix sum of tph over the batch into pre[0..B] (shared memory).
+__device__ void big_build_prefix(const AttnArgs& a, int tpt, int* pre, int* scratch) {
+  const int nt = blockDim.x, tid = threadIdx.x;
+  const int per = (a.B + nt - 1) / nt;
+  const int lo = min(a.B, tid * per), hi = min(a.B, lo + per);
+  int sum = 0;
+  for (int b = lo; b < hi; ++b) {
+    BigSeq s;
+    big_seq(a, b, tpt, s);
+    sum += s.tph;
+  }
+  scratch[tid] = sum;
+  __syncthreads();
+  int base = 0;
+  for (int t = 0; t < tid; ++t) base += scratch[t];
+  for (int b = lo; b < hi; ++b) {
+    BigSeq s;
+    big_seq(a, b, tpt, s);
+    pre[b] = base;
+    base += s.tph;
+  }
+  if (tid == nt - 1) pre[a.B] = base;
+  __syncthreads();
+}
+
+struct BigWalk {
+  BigSeq s;
+  int b, h, rt, ti, tiles_u, tpt;
+  int it, n_iter, piece_idx, piece_j, slot;
+  bool open, first, last;
+  int step_idx, nvalid;     // step_idx < 0: cache tile
+};
+__device__ __forceinline__ void bwalk_init(const AttnArgs& a, BigWalk& w, int tpt, int b0, long long rel,
+                                           int n_iter) {
+  w.tpt = tpt;
+  w.b = b0;
+  big_seq(a, b0, tpt, w.s);
+  w.h = static_cast<int>(rel / w.s.tph);
+  int rem = static_cast<int>(rel - static_cast<long long>(w.h) * w.s.tph);
+  w.rt = 0;
+  for (;;) {
+    const int tu = w.s.cache_tiles + big_step_tiles(w.s, w.rt, tpt);
+    if (rem < tu || w.rt + 1 >= w.s.n_rt) { w.tiles_u = tu; break; }
+    rem -= tu;
+    ++w.rt;
+  }
+  w.ti = rem;
+  w.it = 0;
+  w.n_iter = n_iter;
+  w.piece_idx = -1;
+  w.piece_j = 0;
+  w.slot = 0;
+  w.open = false;
+}
+__device__ __forceinline__ void bwalk_tile(BigWalk& w) {
+  const int left = w.n_iter - w.it;
+  w.first = !w.open;
+  if (w.first) {
+    const bool whole = (w.ti == 0) && (left >= w.tiles_u);
+    w.slot = whole ? -1 : 2 * static_cast<int>(blockIdx.x) + (w.it == 0 ? 0 : 1);
+    w.open = true;
+    w.piece_idx += 1;
+    w.piece_j = 0;
+  }
+  w.step_idx = w.ti - w.s.cache_tiles;
+  w.last = (w.ti == w.tiles_u - 1) || left == 1;
+  w.nvalid = w.step_idx >= 0 ? min(kTile, w.s.n_q - w.step_idx * kTile) : min(kTile, w.s.L - w.ti * kTile);
+}
+__device__ __forceinline__ void bwalk_next(const AttnArgs& a, BigWalk& w) {
+  if (w.last) w.open = false;
+  w.piece_j += 1;
+  w.it += 1;
+  if (++w.ti == w.tiles_u) {
+    w.ti = 0;
+    if (++w.rt == w.s.n_rt) {
+      w.rt = 0;
+      if (++w.h == a.H_kv) {
+        w.h = 0;
+        if (w.it < w.n_iter) {
+          do {
+            ++w.b;
+            big_seq(a, w.b, w.tpt, w.s);
+          } while (w.s.tph == 0 && w.b + 1 < a.B);
+        }
+      }
+    }
+    w.tiles_u = w.s.cache_tiles + big_step_tiles(w.s, w.rt, w.tpt);
+  }
+}
+
+__device__ __host__ inline size_t big_slot_floats() { return static_cast<size_t>(kTile) * (kBD + 2); }
+
+// ---------------------------------------------------------------- kernel
+
+__global__ void __launch_bounds__(kBThreads, 1)
+attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
+                     const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_ks,
+                     const __grid_constant__ CUtensorMap map_vs, const __grid_constant__ CUtensorMap map_q,
+                     int tpt) {
+  constexpr int D = kBD, HALVES = 2, KSTEPS = D / 16;
+  extern __shared__ __align__(1024) uint8_t smem[];
+  const uint32_t sb = smem_u32(smem);
+  const uint32_t bars = sb + kBOffMisc;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kBOffMisc + kBMiscScalars);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kBOffMisc + kBMiscScalars + 8);
+  volatile int* grow_flag = reinterpret_cast<volatile int*>(smem + kBOffMisc + kBMiscScalars + 16);
+  float* s_mx = reinterpret_cast<float*>(smem + kBOffMisc + kBMiscMx);      // [2][128]
+  float* s_lp = reinterpret_cast<float*>(smem + kBOffMisc + kBMiscL);       // [2][128]
+  uint32_t* status = reinterpret_cast<uint32_t*>(a.workspace);
+  int* ws_pre = reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(a.workspace) + kWsHeaderBytes);
+  float* ws_slots = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(a.workspace) + kWsHeaderBytes +
+                                             ws_prefix_bytes());
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (sb & 1023u) {
+    if (threadIdx.x == 0) atomicExch(status, kTimeoutMagic + 1);
+    return;
+  }
+  const int rows_box = tpt * a.G;
+
+  // ---- schedule (the prefix lives where the buffers will be) ----
+  int* s_pre = reinterpret_cast<int*>(smem);
+  int* s_scratch = s_pre + a.B + 1;
+  big_build_prefix(a, tpt, s_pre, s_scratch);
+  const long long n_tiles = static_cast<long long>(s_pre[a.B]) * a.H_kv;
+  const long long t0 = n_tiles * blockIdx.x / gridDim.x;
+  const long long t1 = n_tiles * (blockIdx.x + 1) / gridDim.x;
+  const int n_iter = static_cast<int>(t1 - t0);
+  if (blockIdx.x == 0) {
+    for (int i = threadIdx.x; i <= a.B; i += blockDim.x) ws_pre[i] = s_pre[i];
+  }
+  BigWalk w0;
+  w0.n_iter = 0;
+  if (n_iter > 0) {
+    int lo = 0, hi = a.B;
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (static_cast<long long>(s_pre[mid]) * a.H_kv <= t0) lo = mid; else hi = mid;
+    }
+    bwalk_init(a, w0, tpt, lo, t0 - static_cast<long long>(s_pre[lo]) * a.H_kv, n_iter);
+  }
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kBKv; ++i) {
+      mbar_init(bars + 8 * (kBbKvFull + i), 1);
+      mbar_init(bars + 8 * (kBbKvEmpty + i), 1);
+    }
+    mbar_init(bars + 8 * kBbQFull, 1);
+    mbar_init(bars + 8 * kBbQEmpty, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bars + 8 * (kBbSFull + i), 1);
+      mbar_init(bars + 8 * (kBbPFull + i), 8);
+      mbar_init(bars + 8 * (kBbPvDone + i), 1);
+    }
+    mbar_init(bars + 8 * kBbAll, 8);
+    mbar_init(bars + 8 * kBbDrain, 1);
+    *abort_flag = 0;
+    *grow_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();   // the prefix has been consumed
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                     smem_u32(tmem_slot)), "r"(kBCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  if (warp == 0 && lane == 0 && n_iter > 0) {
+    // =========================== TMA producer ===========================
+    BigWalk w = w0;
+    bool ok = true;
+    int uses = 0, pieces = 0;
+    RingPos rp;
+    rp.init(0, kBKv);
+    while (w.it < n_iter) {
+      bwalk_tile(w);
+      if (w.first) {
+        // one Q buffer: every Q K^T of the previous unit must have read it
+        if (!mbar_wait(bars + 8 * kBbQEmpty, (w.piece_idx & 1) ^ 1, abort_flag, status)) { ok = false; break; }
+        fence_async_smem();
+        const uint32_t bar = bars + 8 * kBbQFull;
+        mbar_arrive_expect_tx(bar, static_cast<uint32_t>(HALVES * rows_box * 128));
+#pragma unroll
+        for (int hf = 0; hf < HALVES; ++hf)
+          tma_load_3d(sb + kBOffQ + hf * kBHalf, &map_q, bar, hf * 64, w.h * a.G, w.s.r0 + w.rt * tpt);
+        ++pieces;
+      }
+#pragma unroll 1
+      for (int kv = 0; kv < 2; ++kv) {
+        const int buf = rp.buf;
+        if (!mbar_wait(bars + 8 * (kBbKvEmpty + buf), rp.par ^ 1u, abort_flag, status)) { ok = false; break; }
+        rp.step(1);
+        fence_async_smem();
+        const uint32_t dst = sb + kBOffKv + buf * kBKvBytes;
+        const uint32_t bar = bars + 8 * (kBbKvFull + buf);
+        mbar_arrive_expect_tx(bar, static_cast<uint32_t>(kBKvBytes));
+        if (w.step_idx >= 0) {
+          const int z = w.s.r0 + w.step_idx * kTile;
+#pragma unroll
+          for (int hf = 0; hf < HALVES; ++hf)
+            tma_load_3d(dst + hf * kBHalf, kv ? &map_vs : &map_ks, bar, hf * 64, w.h, z);
+        } else {
+          const int y = static_cast<int>(w.s.slot_off) + w.ti * kTile;
+#pragma unroll
+          for (int hf = 0; hf < HALVES; ++hf)
+            tma_load_3d(dst + hf * kBHalf, kv ? &map_v : &map_k, bar, hf * 64, y, w.h);
+        }
+        ++uses;
+      }
+      if (!ok) break;
+      bwalk_next(a, w);
+    }
+    for (int u = uses > kBKv ? uses - kBKv : 0; u < uses; ++u)
+      (void)mbar_wait(bars + 8 * (kBbKvFull + u % kBKv), (u / kBKv) & 1, abort_flag, status);
+    if (pieces > 0) (void)mbar_wait(bars + 8 * kBbQFull, (pieces - 1) & 1, abort_flag, status);
+  } else if (warp == 1 && lane == 0 && n_iter > 0) {
+    // =========================== MMA issuer ===========================
+    const uint32_t idesc_qk = instr_desc(kTile, 0), idesc_pv = instr_desc(D, 1);
+    const uint32_t q_lo = desc_lo(sb + kBOffQ, 16), k_lo0 = desc_lo(sb + kBOffKv, 16);
+    const uint32_t p_lo0 = desc_lo(sb + kBOffP, 16), v_lo0 = desc_lo(sb + kBOffKv, kBHalf);
+    BigWalk wq = w0, wp = w0;
+    RingPos rk, rv;
+    rk.init(0, kBKv);
+    rv.init(1, kBKv);
+    bool ok = true;
+    auto issue_qk = [&]() -> bool {
+      bwalk_tile(wq);
+      const int it = wq.it;
+      if ((wq.first && !mbar_wait(bars + 8 * kBbQFull, wq.piece_idx & 1, abort_flag, status)) ||
+          !mbar_wait(bars + 8 * (kBbKvFull + rk.buf), rk.par, abort_flag, status))
+        return false;
+      tc_fence_after();
+      const uint32_t k_lo = k_lo0 + rk.buf * (kBKvBytes >> 4);
+      const uint32_t d_s = tmem + kBColS + (it & 1) * kTile;
+#pragma unroll
+      for (int ks = 0; ks < KSTEPS; ++ks) {
+        const uint32_t off = (ks >> 2) * (kBHalf >> 4) + (ks & 3) * 2;
+        umma_bf16_lo(d_s, q_lo + off, k_lo + off, idesc_qk, ks > 0);
+      }
+      umma_commit(bars + 8 * (kBbKvEmpty + rk.buf));
+      umma_commit(bars + 8 * (kBbSFull + (it & 1)));
+      if (wq.last) umma_commit(bars + 8 * kBbQEmpty);
+      rk.step(2);
+      bwalk_next(a, wq);
+      return true;
+    };
+    ok = issue_qk();
+    while (ok && wp.it < n_iter) {
+      if (wq.it < n_iter && !issue_qk()) { ok = false; break; }
+      bwalk_tile(wp);
+      const int it = wp.it;
+      if (!mbar_wait(bars + 8 * (kBbPFull + (it & 1)), (it >> 1) & 1, abort_flag, status) ||
+          !mbar_wait(bars + 8 * (kBbKvFull + rv.buf), rv.par, abort_flag, status)) {
+        ok = false;
+        break;
+      }
+      tc_fence_after();
+      const uint32_t p_lo = p_lo0 + (it & 1) * (kBPBytes >> 4);
+      const uint32_t v_lo = v_lo0 + rv.buf * (kBKvBytes >> 4);
+      const int ksteps = (wp.nvalid + 15) >> 4;
+      const uint32_t acc0 = wp.first ? 0u : 1u;
+      if (ksteps == kTile / 16) {
+#pragma unroll
+        for (int j = 0; j < kTile / 16; ++j)
+          umma_bf16_lo(tmem + kBColO, p_lo + (j >> 2) * (kBHalf >> 4) + (j & 3) * 2, v_lo + j * (2048 >> 4),
+                       idesc_pv, j == 0 ? acc0 : 1u);
+      } else {
+#pragma unroll 1
+        for (int j = 0; j < ksteps; ++j)
+          umma_bf16_lo(tmem + kBColO, p_lo + (j >> 2) * (kBHalf >> 4) + (j & 3) * 2, v_lo + j * (2048 >> 4),
+                       idesc_pv, j == 0 ? acc0 : 1u);
+      }
+      umma_commit(bars + 8 * (kBbKvEmpty + rv.buf));
+      umma_commit(bars + 8 * (kBbPvDone + (it & 1)));
+      rv.step(2);
+      bwalk_next(a, wp);
+    }
+    if (!ok) {
+      umma_commit(bars + 8 * kBbDrain);
+      const unsigned long long t_begin = global_ns();
+      while (!mbar_try_wait(bars + 8 * kBbDrain, 0) && global_ns() - t_begin < kWaitLimitNs) {
+      }
+    }
+  } else if (warp >= 4 && n_iter > 0) {
+    // ====== softmax warps: thread = packed row; warpgroup g = key columns / output columns [64g, 64g+64) ======
+    const int wg = (warp - 4) >> 2, quad = (warp - 4) & 3;
+    const int r = quad * 32 + lane;
+    const uint32_t lane_addr = tmem + (static_cast<uint32_t>(quad * 32) << 16);
+    const uint32_t rx = r & 7;
+    BigWalk w = w0;
+    float m_ref = 0.f, l_part = 0.f;
+    int tok = 0, anc = 0, rows = 0;
+    bool row_ok = false;
+    uint32_t all_phase = 0;
+    bool ok = true;
+    auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {
+      return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, status));
+    };
+    // bounded barrier of the eight softmax warps (also publishes their shared-memory writes)
+    auto sync8 = [&]() -> bool {
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bars + 8 * kBbAll);
+      const bool good = wait_all(bars + 8 * kBbAll, all_phase & 1);
+      ++all_phase;
+      return good;
+    };
+    while (ok && w.it < n_iter) {
+      bwalk_tile(w);
+      const int it = w.it, pb = it & 1;
+      if (w.first) {
+        const int tok0 = w.rt * tpt;
+        rows = (min(w.s.n_q, tok0 + tpt) - tok0) * a.G;
+        row_ok = r < rows;
+        if (row_ok) {
+          const int i = tok0 + r / a.G;
+          tok = i;
+          anc = (i < w.s.n_c) ? i : (a.anchor ? a.anchor[w.s.r0 + i] : w.s.n_c);
+        } else {
+          tok = 1 << 20;
+          anc = 0;
+        }
+      }
+      if (!wait_all(bars + 8 * (kBbSFull + pb), (it >> 1) & 1)) { ok = false; break; }
+      if (it >= 2 && !wait_all(bars + 8 * (kBbPvDone + pb), ((it >> 1) - 1) & 1)) { ok = false; break; }
+      tc_fence_after();
+      const int nv = w.nvalid;
+      const bool is_step = w.step_idx >= 0;
+      const bool masked = is_step || nv < kTile;
+      if (masked && (nv & 15)) {
+        // V rows past the valid keys hold foreign or stale bytes; P is 0 there but 0 * NaN is NaN
+        const int use = 2 * it + 1, buf = use % kBKv;
+        if (!wait_all(bars + 8 * (kBbKvFull + buf), (use / kBKv) & 1)) { ok = false; break; }
+        const uint32_t va = sb + kBOffKv + buf * kBKvBytes;
+        const int n_rows = ((nv + 15) & ~15) - nv;
+        for (int x = wg * 128 + r; x < n_rows * HALVES * 8; x += 256) {
+          const int rr = nv + x / (HALVES * 8), cc = x % (HALVES * 8);
+          const uint32_t addr = va + (cc >> 3) * kBHalf + rr * 128 + ((cc & 7) << 4);
+          asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(addr), "r"(0u) : "memory");
+        }
+      }
+      // this warpgroup's 64 score columns of the row; invisible keys become -inf
+      const uint32_t s_addr = lane_addr + kBColS + pb * kTile + wg * 64;
+      const int key0 = (is_step ? w.step_idx * kTile : 0) + wg * 64;   // step-local index of column 0
+      float v[64];
+      auto load_scores = [&]() {
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          uint32_t raw[32];
+          tmem_ld32(s_addr + c * 32, raw);
+          tmem_ld_wait(raw);
+#pragma unroll
+          for (int e = 0; e < 32; ++e) {
+            float s = __uint_as_float(raw[e]);
+            if (masked) {
+              const int col = wg * 64 + c * 32 + e;
+              bool vis = col < nv;
+              if (is_step) vis = vis && step_key_visible(tok, key0 + c * 32 + e, w.s.n_c, anc);
+              s = vis ? s : -INFINITY;
+            }
+            v[c * 32 + e] = s;
+          }
+        }
+      };
+      auto row_max = [&]() -> float {
+        float m = -INFINITY;
+#pragma unroll
+        for (int j = 0; j < 64; ++j) m = fmaxf(m, v[j]);
+        return m;
+      };
+      load_scores();
+      if (w.piece_j == 0) {
+        // new unit: reference = exact maximum of the first tile over both column halves
+        s_mx[wg * 128 + r] = row_max();
+        if (!sync8()) { ok = false; break; }
+        const float m = fmaxf(s_mx[r], s_mx[128 + r]);
+        m_ref = (m == -INFINITY) ? 0.f : m * a.scale_log2;
+        l_part = 0.f;
+      }
+      float tmaxx = -INFINITY;
+#pragma unroll
+      for (int j = 0; j < 64; ++j) {
+        v[j] = fmaf(v[j], a.scale_log2, -m_ref);
+        tmaxx = fmaxf(tmaxx, v[j]);
+      }
+      if (w.piece_j > 0 && __any_sync(0xffffffffu, row_ok && tmaxx > kBGrowLimit) && lane == 0)
+        *grow_flag = it + 1;
+      if (!sync8()) { ok = false; break; }
+      if (*grow_flag == it + 1) {
+        // ---- rare: move the row references up; rescale O (this group's 64 columns) and the sums ----
+        load_scores();
+        s_mx[wg * 128 + r] = row_max();
+        if (!sync8()) { ok = false; break; }
+        const float m = fmaxf(s_mx[r], s_mx[128 + r]);
+        const float m_new = (m == -INFINITY) ? m_ref : fmaxf(m_ref, m * a.scale_log2);
+        const float alpha = ex2(m_ref - m_new);
+        m_ref = m_new;
+        l_part *= alpha;
+        if (!wait_all(bars + 8 * (kBbPvDone + ((it - 1) & 1)), ((it - 1) >> 1) & 1)) { ok = false; break; }
+        tc_fence_after();
+#pragma unroll 1
+        for (int c = 0; c < 2; ++c) {
+          uint32_t o[32];
+          tmem_ld32(lane_addr + kBColO + wg * 64 + c * 32, o);
+          tmem_ld_wait(o);
+#pragma unroll
+          for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+          tmem_st32(lane_addr + kBColO + wg * 64 + c * 32, o);
+        }
+        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+#pragma unroll
+        for (int j = 0; j < 64; ++j) v[j] = fmaf(v[j], a.scale_log2, -m_ref);
+        if (!sync8()) { ok = false; break; }     // s_mx may be rewritten from here on
+      }
+      // p = 2^x as bf16 into this row of the P tile (half g = this group's 64 keys)
+      {
+        const uint32_t p_row = sb + kBOffP + pb * kBPBytes + wg * kBHalf + r * 128;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          float p[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            p[e] = ex2(v[c * 8 + e]);
+            l_part += p[e];
+          }
+          const uint32_t addr = p_row + ((c ^ rx) << 4);
+          asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(pack2(p[0], p[1])),
+                       "r"(pack2(p[2], p[3])), "r"(pack2(p[4], p[5])), "r"(pack2(p[6], p[7]))
+                       : "memory");
+        }
+      }
+      fence_async_smem();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bars + 8 * (kBbPFull + pb));
+
+      if (w.last) {
+        // ---- end of the unit (or of this CTA's part of it) ----
+        s_lp[wg * 128 + r] = l_part;
+        if (!sync8()) { ok = false; break; }
+        const float l_row = s_lp[r] + s_lp[128 + r];
+        if (!wait_all(bars + 8 * (kBbPvDone + pb), (it >> 1) & 1)) { ok = false; break; }
+        tc_fence_after();
+        const int i = tok, g = r % a.G;
+        const int64_t orow = static_cast<int64_t>(w.s.r0 + (row_ok ? i : 0)) * a.H_q + w.h * a.G + g;
+        float* slot = ws_slots + static_cast<size_t>(w.slot < 0 ? 0 : w.slot) * big_slot_floats();
+        const float inv = 1.f / l_row;
+#pragma unroll 1
+        for (int c = 0; c < 2; ++c) {
+          uint32_t o[32];
+          tmem_ld32(lane_addr + kBColO + wg * 64 + c * 32, o);
+          tmem_ld_wait(o);
+          if (row_ok && w.slot < 0) {
+            uint4* op = reinterpret_cast<uint4*>(a.out + orow * D + wg * 64 + c * 32);
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4) {
+              uint4 u;
+              u.x = pack2(__uint_as_float(o[8 * q4 + 0]) * inv, __uint_as_float(o[8 * q4 + 1]) * inv);
+              u.y = pack2(__uint_as_float(o[8 * q4 + 2]) * inv, __uint_as_float(o[8 * q4 + 3]) * inv);
+              u.z = pack2(__uint_as_float(o[8 * q4 + 4]) * inv, __uint_as_float(o[8 * q4 + 5]) * inv);
+              u.w = pack2(__uint_as_float(o[8 * q4 + 6]) * inv, __uint_as_float(o[8 * q4 + 7]) * inv);
+              op[q4] = u;
+            }
+          } else if (row_ok) {
+            uint4* sp = reinterpret_cast<uint4*>(slot + static_cast<size_t>(r) * D + wg * 64 + c * 32);
+#pragma unroll
+            for (int q4 = 0; q4 < 8; ++q4) sp[q4] = make_uint4(o[4 * q4], o[4 * q4 + 1], o[4 * q4 + 2], o[4 * q4 + 3]);
+          }
+        }
+        if (row_ok && wg == 0) {
+          if (w.slot < 0) {
+            if (a.lse) a.lse[orow] = (m_ref + log2f(l_row)) * 0.69314718055994531f;
+          } else {
+            float* sm = slot + static_cast<size_t>(kTile) * D;
+            sm[r] = m_ref;
+            sm[kTile + r] = l_row;
+          }
+        }
+        tc_fence_before();   // the reads of O are ordered before the next unit's first PV product
+      }
+      bwalk_next(a, w);
+    }
+  }
+
+  // ---- teardown: every thread arrives here, on success and on abort ----
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    __syncwarp();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kBCols) : "memory");
+  }
+}
+
+// One CTA per (sequence, KV head, row tile) unit that the split kernel cut across CTAs; one warp
+// per packed row folds the pieces' (m, l) with shuffles and accumulates its output columns.
+__global__ void __launch_bounds__(128)
+attn_big_merge_kernel(const AttnArgs a, int tpt, int max_rt, int n_ctas) {
+  constexpr int D = kBD, E = D / 32;
+  int u = blockIdx.x;
+  const int rt = u % max_rt; u /= max_rt;
+  const int h = u % a.H_kv;
+  const int b = u / a.H_kv;
+  const int* ws_pre = reinterpret_cast<const int*>(reinterpret_cast<const uint8_t*>(a.workspace) +
+                                                   kWsHeaderBytes);
+  const float* ws_slots = reinterpret_cast<const float*>(
+      reinterpret_cast<const uint8_t*>(a.workspace) + kWsHeaderBytes + ws_prefix_bytes());
+  BigSeq s;
+  big_seq(a, b, tpt, s);
+  if (rt >= s.n_rt || s.tph == 0) return;
+  const long long n_tiles = static_cast<long long>(ws_pre[a.B]) * a.H_kv;
+  long long u0 = static_cast<long long>(ws_pre[b]) * a.H_kv + static_cast<long long>(h) * s.tph;
+  for (int x = 0; x < rt; ++x) u0 += s.cache_tiles + big_step_tiles(s, x, tpt);
+  const long long u1 = u0 + s.cache_tiles + big_step_tiles(s, rt, tpt);
+  const int c_lo = static_cast<int>(((u0 + 1) * n_ctas - 1) / n_tiles);
+  const int c_hi = static_cast<int>((u1 * n_ctas - 1) / n_tiles);
+  if (c_lo == c_hi) return;                      // whole unit inside one CTA: already written
+  const int tok0 = rt * tpt;
+  const int rows = (min(s.n_q, tok0 + tpt) - tok0) * a.G;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const size_t slot_floats = big_slot_floats();
+  for (int r = warp; r < rows; r += 4) {
+    float M = -INFINITY;
+    for (int c = c_lo + lane; c <= c_hi; c += 32) {
+      const long long s0 = n_tiles * c / n_ctas, s1 = n_tiles * (c + 1) / n_ctas;
+      if (s1 <= s0) continue;
+      const int slot = 2 * c + ((s0 >= u0) ? 0 : 1);
+      M = fmaxf(M, ws_slots[slot * slot_floats + static_cast<size_t>(kTile) * D + r]);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+    float Lsum = 0.f, acc[E];
+#pragma unroll
+    for (int e = 0; e < E; ++e) acc[e] = 0.f;
+    for (int c = c_lo; c <= c_hi; ++c) {
+      const long long s0 = n_tiles * c / n_ctas, s1 = n_tiles * (c + 1) / n_ctas;
+      if (s1 <= s0) continue;
+      const int slot = 2 * c + ((s0 >= u0) ? 0 : 1);
+      const float* sp = ws_slots + slot * slot_floats;
+      const float m = sp[static_cast<size_t>(kTile) * D + r];
+      const float l = sp[static_cast<size_t>(kTile) * D + kTile + r];
+      const float wgt = (m == -INFINITY) ? 0.f : exp2f(m - M);
+      Lsum += l * wgt;
+      const float* po = sp + static_cast<size_t>(r) * D + lane * E;
+#pragma unroll
+      for (int e = 0; e < E; ++e) acc[e] += wgt * po[e];
+    }
+    const int i = tok0 + r / a.G, g = r % a.G;
+    const int64_t orow = static_cast<int64_t>(s.r0 + i) * a.H_q + h * a.G + g;
+    const float inv = 1.f / Lsum;
+    __nv_bfloat16* op = a.out + orow * D + lane * E;
+#pragma unroll
+    for (int e = 0; e < E; e += 2) *reinterpret_cast<uint32_t*>(op + e) = pack2(acc[e] * inv, acc[e + 1] * inv);
+    if (a.lse && lane == 0) a.lse[orow] = (M + log2f(Lsum)) * 0.69314718055994531f;
+  }
+}
+
+}  // namespace
+
+bool attn_umma_big_supports(int D, int G, int max_nq) {
+  return D == kBD && G >= 1 && G <= kMaxGroup && max_nq > kMaxNq && max_nq <= kMaxNqBig;
+}
+
+size_t attn_umma_big_workspace_bytes(int n_ctas) {
+  return kWsHeaderBytes + ws_prefix_bytes() + static_cast<size_t>(2) * n_ctas * big_slot_floats() * sizeof(float);
+}
+
+int32_t launch_attn_umma_big(const AttnArgs& a, cudaStream_t st) {
+  if (a.B == 0 || a.T == 0) return MS_OK;
+  if (!attn_umma_big_supports(a.D, a.G, a.max_nq)) return MS_ERR_UNSUPPORTED_SHAPE;
+  if (static_cast<int>((a.B + 1 + kBThreads) * sizeof(int)) > kBOffMisc) return MS_ERR_UNSUPPORTED_SHAPE;
+  const int tpt = kTile / a.G;                   // tokens per row tile
+  const int max_rt = (a.max_nq + tpt - 1) / tpt;
+  const int grid = attn_mma_grid();
+  if (grid <= 0) return cuda_status(cudaErrorNoDevice);
+  CUtensorMap mk, mv, mks, mvs, mq;
+  const bool ok =
+      make_map(&mk, a.k_cache, a.D, static_cast<uint64_t>(a.n_slots), a.H_kv, a.D, a.kv_head_stride, kTile, 1) &&
+      make_map(&mv, a.v_cache, a.D, static_cast<uint64_t>(a.n_slots), a.H_kv, a.D, a.kv_head_stride, kTile, 1) &&
+      make_map(&mks, a.k_step, a.D, a.H_kv, a.T, a.D, static_cast<uint64_t>(a.H_kv) * a.D, 1, kTile) &&
+      make_map(&mvs, a.v_step, a.D, a.H_kv, a.T, a.D, static_cast<uint64_t>(a.H_kv) * a.D, 1, kTile) &&
+      make_map(&mq, a.q, a.D, a.H_q, a.T, a.D, static_cast<uint64_t>(a.H_q) * a.D, a.G, tpt);
+  if (!ok) return cuda_status(cudaErrorInvalidValue);
+  static bool configured[64] = {false};
+  int dev = 0;
+  MS_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev >= 0 && dev < 64 && !configured[dev]) {
+    MS_CUDA_TRY(cudaFuncSetAttribute(attn_umma_big_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kBSmem));
+    configured[dev] = true;
+  }
+  if (a.ev_split_begin) MS_CUDA_TRY(cudaEventRecord(a.ev_split_begin, st));
+  attn_umma_big_kernel<<<grid, kBThreads, kBSmem, st>>>(a, mk, mv, mks, mvs, mq, tpt);
+  MS_LAUNCH_CHECK();
+  if (a.ev_split_end) MS_CUDA_TRY(cudaEventRecord(a.ev_split_end, st));
+  const long long units = static_cast<long long>(a.B) * a.H_kv * max_rt;
+  attn_big_merge_kernel<<<static_cast<unsigned>(units), 128, 0, st>>>(a, tpt, max_rt, grid);
+  MS_LAUNCH_CHECK();
+  return MS_OK;
+}
+
+}  // namespace ms

@@ -572,7 +572,7 @@ int32_t launch_t(const AttnArgs& a, cudaStream_t st, int rows_pad, int grid, con
 
 }  // namespace
 
-bool attn_umma_t_supports(int D, int G, int max_nq) { return D == 128 && G * max_nq <= 64; }
+bool attn_umma_t_supports(int D, int G, int max_nq) { return D == 128 && max_nq <= kMaxNq && G * max_nq <= 64; }
 
 int32_t launch_attn_umma_t(const AttnArgs& a, cudaStream_t st) {
   if (a.B == 0 || a.T == 0) return MS_OK;

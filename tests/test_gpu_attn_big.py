@@ -1,0 +1,86 @@
+"""GPU parity of the large-block attention (17..256 new tokens per sequence): the compression
+pass of the method forwards the l memory tokens and <o> of a finished reasoning step as one
+causal block against the compacted cache (Sec. 2.1.2; Algorithm 1).  Same call
+(memosight_attn_step, max_nq > 16), same oracle, same tolerance as the step blocks."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from conftest import bits
+from harness import check_attn, gpu_attn, oracle_attn, random_problem
+from paper_2604_14889_b200 import binding as ms
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("name,kw", [
+    ("G4 one row tile and a bit", dict(B=1, Hq=4, Hkv=1, D=128, lens=[300], n_q_list=[40], n_c_list=[40], seed=1)),
+    ("AMA(512,3)+1 tokens", dict(B=2, Hq=8, Hkv=2, D=128, lens=[1000, 77], n_q_list=[172, 33], n_c_list=[172, 20],
+                                 seed=2, anchors=True)),
+    ("G7: 18 tokens per row tile", dict(B=2, Hq=28, Hkv=4, D=128, lens=[513, 128], n_q_list=[50, 17],
+                                        n_c_list=[50, 17], seed=3)),
+    ("G1: two step-key tiles", dict(B=1, Hq=2, Hkv=2, D=128, lens=[700], n_q_list=[200], n_c_list=[200], seed=4)),
+    ("G16: 8 tokens per row tile", dict(B=1, Hq=16, Hkv=1, D=128, lens=[257], n_q_list=[20], n_c_list=[12], seed=5,
+                                        anchors=True)),
+    ("empty cache", dict(B=1, Hq=8, Hkv=2, D=128, lens=[0], n_q_list=[172], n_c_list=[172], seed=6)),
+    ("long cache, units cut across CTAs", dict(B=1, Hq=32, Hkv=8, D=128, lens=[20000], n_q_list=[172],
+                                               n_c_list=[172], seed=7)),
+    ("small, large, empty and maximal blocks", dict(B=4, Hq=8, Hkv=2, D=128, lens=[900, 5000, 0, 130],
+                                                    n_q_list=[3, 172, 0, 256], n_c_list=[2, 172, 0, 100], seed=8,
+                                                    anchors=True)),
+    ("peaked scores", dict(B=2, Hq=8, Hkv=2, D=128, lens=[3000, 640], n_q_list=[100, 64], n_c_list=[100, 64], seed=9,
+                           qscale=6.0)),
+])
+def test_large_blocks_match_oracle(name, kw):
+    check_attn(random_problem(**kw), name)
+
+
+def test_large_block_reference_moves_and_garbage_tail():
+    P = random_problem(2, 8, 2, 128, [148 * 128 + 50, 300], [172, 40], [172, 40], seed=31, headroom=150)
+    r0 = int(P["q_off"][0])
+    q = P["q"][r0 + 100, 5].float()                       # token 100, head 5 -> KV head 1
+    for pos, strength in ((200, 45.0), (9000, 100.0)):    # > 2^48 above everything before, twice
+        P["k_cache"][1, int(P["kv_off"][0]) + pos] = (strength * np.sqrt(128) * q / q.norm() ** 2).to(torch.bfloat16)
+    q2 = P["q"][r0 + 150, 0].float()                      # a step-local needle: key 140 seen by token 150
+    P["k_step"][r0 + 140, 0] = (60.0 * np.sqrt(128) * q2 / q2.norm() ** 2).to(torch.bfloat16)
+    want, want_lse = oracle_attn(P)
+    for b in range(2):
+        lo = int(P["kv_off"][b]) + P["lens"][b]
+        P["k_cache"][:, lo:lo + 150] = float("nan")
+        P["v_cache"][:, lo:lo + 150] = float("inf")
+    out, lse = gpu_attn(P)
+    from harness import assert_attn_close
+    assert_attn_close(out, lse, want, want_lse, "needles + garbage tail")
+
+
+def test_large_block_equals_the_same_tokens_as_small_blocks():
+    # a causal block of 32 tokens gives, row for row, what two causal blocks of 16 give when the
+    # first 16 tokens have been appended to the cache in between (ties the large-block kernel to
+    # the step kernels and to kv_append)
+    dev = "cuda"
+    P = random_problem(1, 8, 2, 128, [500], [32], [32], seed=41, headroom=40)
+    big, _ = gpu_attn(P)
+    Hkv, D, stride = 2, 128, P["n_slots"] * 128
+    kc, vc = P["k_cache"].to(dev).clone(), P["v_cache"].to(dev).clone()
+    kv_len = P["kv_len"].to(dev).clone()
+    first = dict(P, T=16, max_nq=16, q=P["q"][:16], k_step=P["k_step"][:16], v_step=P["v_step"][:16],
+                 q_off=torch.tensor([0, 16], dtype=torch.int32), n_cand=torch.tensor([16], dtype=torch.int32))
+    out1, _ = gpu_attn(first)
+    ms.memosight_kv_append(kc, vc, stride, 1, Hkv, D, P["kv_off"].to(dev), kv_len, P["k_step"][:16].to(dev),
+                           P["v_step"][:16].to(dev), first["q_off"].to(dev), first["n_cand"].to(dev),
+                           torch.tensor([16], dtype=torch.int32, device=dev), 16, 1)
+    torch.cuda.synchronize()
+    second = dict(first, k_cache=kc.cpu(), v_cache=vc.cpu(), kv_len=kv_len.cpu(), lens=[516], q=P["q"][16:],
+                  k_step=P["k_step"][16:], v_step=P["v_step"][16:])
+    out2, _ = gpu_attn(second)
+    assert (big[:16].float() - out1.float()).abs().max() <= 2e-2
+    assert (big[16:].float() - out2.float()).abs().max() <= 2e-2
+
+
+def test_block_size_limits():
+    P = random_problem(1, 8, 2, 128, [10], [16], [16], seed=1)
+    assert ms.memosight_attn_workspace_bytes(1, 8, 2, 128, 10, 257) == 0
+    assert ms.memosight_attn_workspace_bytes(1, 8, 2, 128, 10, 256) > ms.memosight_attn_workspace_bytes(1, 8, 2, 128, 10, 16)
+    # head_dim 64 has no large-block tensor-core kernel: the general kernel serves it
+    check_attn(random_problem(1, 4, 2, 64, [200], [40], [40], seed=2), "D=64 large block")
