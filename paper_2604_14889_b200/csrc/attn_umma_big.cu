@@ -159,6 +159,38 @@ __device__ __forceinline__ void bwalk_next(const AttnArgs& a, BigWalk& w) {
 
 __device__ __host__ inline size_t big_slot_floats() { return static_cast<size_t>(kTile) * (kBD + 2); }
 
+// The warpgroup's 64 score columns of one row, from tensor memory into v[]; with kMasked the
+// invisible keys (past the valid length; on a step-local tile by the (n_cand, anchor) rule)
+// become -inf.
+template <bool kMasked>
+__device__ __forceinline__ void big_load_scores(uint32_t s_addr, float (&v)[64], int col0, int nv, bool is_step,
+                                                int tok, int key0, int n_c, int anc) {
+#pragma unroll
+  for (int c = 0; c < 2; ++c) {
+    uint32_t raw[32];
+    tmem_ld32(s_addr + c * 32, raw);
+    tmem_ld_wait(raw);
+#pragma unroll
+    for (int e = 0; e < 32; ++e) {
+      float s = __uint_as_float(raw[e]);
+      if (kMasked) {
+        bool vis = col0 + c * 32 + e < nv;
+        if (is_step) vis = vis && step_key_visible(tok, key0 + c * 32 + e, n_c, anc);
+        s = vis ? s : -INFINITY;
+      }
+      v[c * 32 + e] = s;
+    }
+  }
+}
+__device__ __forceinline__ float max64(const float (&v)[64]) {
+  float m[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) m[j] = v[j];
+#pragma unroll
+  for (int j = 8; j < 64; ++j) m[j & 7] = fmaxf(m[j & 7], v[j]);
+  return fmaxf(fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3])), fmaxf(fmaxf(m[4], m[5]), fmaxf(m[6], m[7])));
+}
+
 // ---------------------------------------------------------------- kernel
 
 __global__ void __launch_bounds__(kBThreads, 1)
@@ -415,52 +447,30 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
       const int key0 = (is_step ? w.step_idx * kTile : 0) + wg * 64;   // step-local index of column 0
       float v[64];
       auto load_scores = [&]() {
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          uint32_t raw[32];
-          tmem_ld32(s_addr + c * 32, raw);
-          tmem_ld_wait(raw);
-#pragma unroll
-          for (int e = 0; e < 32; ++e) {
-            float s = __uint_as_float(raw[e]);
-            if (masked) {
-              const int col = wg * 64 + c * 32 + e;
-              bool vis = col < nv;
-              if (is_step) vis = vis && step_key_visible(tok, key0 + c * 32 + e, w.s.n_c, anc);
-              s = vis ? s : -INFINITY;
-            }
-            v[c * 32 + e] = s;
-          }
-        }
-      };
-      auto row_max = [&]() -> float {
-        float m = -INFINITY;
-#pragma unroll
-        for (int j = 0; j < 64; ++j) m = fmaxf(m, v[j]);
-        return m;
+        if (masked)
+          big_load_scores<true>(s_addr, v, wg * 64, nv, is_step, tok, key0, w.s.n_c, anc);
+        else
+          big_load_scores<false>(s_addr, v, 0, kTile, false, 0, 0, 0, 0);
       };
       load_scores();
       if (w.piece_j == 0) {
         // new unit: reference = exact maximum of the first tile over both column halves
-        s_mx[wg * 128 + r] = row_max();
+        s_mx[wg * 128 + r] = max64(v);
         if (!sync8()) { ok = false; break; }
         const float m = fmaxf(s_mx[r], s_mx[128 + r]);
         m_ref = (m == -INFINITY) ? 0.f : m * a.scale_log2;
         l_part = 0.f;
       }
-      float tmaxx = -INFINITY;
 #pragma unroll
-      for (int j = 0; j < 64; ++j) {
-        v[j] = fmaf(v[j], a.scale_log2, -m_ref);
-        tmaxx = fmaxf(tmaxx, v[j]);
-      }
+      for (int j = 0; j < 64; ++j) v[j] = fmaf(v[j], a.scale_log2, -m_ref);
+      const float tmaxx = max64(v);
       if (w.piece_j > 0 && __any_sync(0xffffffffu, row_ok && tmaxx > kBGrowLimit) && lane == 0)
         *grow_flag = it + 1;
       if (!sync8()) { ok = false; break; }
       if (*grow_flag == it + 1) {
         // ---- rare: move the row references up; rescale O (this group's 64 columns) and the sums ----
         load_scores();
-        s_mx[wg * 128 + r] = row_max();
+        s_mx[wg * 128 + r] = max64(v);
         if (!sync8()) { ok = false; break; }
         const float m = fmaxf(s_mx[r], s_mx[128 + r]);
         const float m_new = (m == -INFINITY) ? m_ref : fmaxf(m_ref, m * a.scale_log2);
@@ -487,18 +497,21 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
       {
         const uint32_t p_row = sb + kBOffP + pb * kBPBytes + wg * kBHalf + r * 128;
 #pragma unroll
+        float ls[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
         for (int c = 0; c < 8; ++c) {
           float p[8];
 #pragma unroll
           for (int e = 0; e < 8; ++e) {
             p[e] = ex2(v[c * 8 + e]);
-            l_part += p[e];
+            ls[e & 3] += p[e];
           }
           const uint32_t addr = p_row + ((c ^ rx) << 4);
           asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(pack2(p[0], p[1])),
                        "r"(pack2(p[2], p[3])), "r"(pack2(p[4], p[5])), "r"(pack2(p[6], p[7]))
                        : "memory");
         }
+        l_part += (ls[0] + ls[1]) + (ls[2] + ls[3]);
       }
       fence_async_smem();
       tc_fence_before();
