@@ -61,6 +61,9 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample-seqs", type=int, default=32)
+    ap.add_argument("--workload", default="step", choices=["step", "compress"],
+                    help="step: the Predict+Verify step the headline metric is quoted on (default); "
+                         "compress: the compression event (forward of the memory tokens + <o>, append, eviction)")
     ap.add_argument("--attn-path", default="auto", choices=["auto", "mma_sync", "tcgen05", "tcgen05_keys"],
                     help="attention kernel: by shape (default), or forced for A/B timing")
     return ap.parse_args()
@@ -297,6 +300,9 @@ def main():
     ms.memosight_attn_set_path({"auto": ms.MS_ATTN_PATH_AUTO, "mma_sync": ms.MS_ATTN_PATH_MMA_SYNC,
                                 "tcgen05": ms.MS_ATTN_PATH_TCGEN05,
                                 "tcgen05_keys": ms.MS_ATTN_PATH_TCGEN05_KEYS}[args.attn_path])
+    if args.workload == "compress":
+        run_compress(args, ms, dev, world, rank)
+        return
     K, W = args.steps, max(args.warmup, 3)
     cfg0 = synth.sweep(args.batch, args.d, args.kv_len, True)
     n_e2e = 0 if args.no_e2e else max(1, min(args.e2e_steps, K))
@@ -433,6 +439,107 @@ def main():
         import torch.distributed as dist
         dist.barrier()
         dist.destroy_process_group()
+
+
+def peak_tensor():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            j = json.load(f)
+        return float(j["bf16_tflops_sustained"]), float(j["bf16_tflops"]), "measured"
+    except Exception:
+        return 1400.0, 1590.0, "fallback"
+
+
+def run_compress(args, ms, dev, world, rank):
+    """Secondary workload: the compression event of long-CoT serving.  Every sequence has just
+    finished a 512-token reasoning step; the 170 memory tokens + <o> are forwarded as one causal
+    block against the cache (which still holds the verbose step), appended, and the step is
+    evicted.  One "step" = that event for the whole batch, one layer.  Compute-bound: the
+    roofline is the bf16 tensor peak."""
+    assert world == 1, "the compress workload is a single-GPU measurement"
+    K, W = args.steps, max(args.warmup, 3)
+    B = args.batch if args.batch != 128 else 16
+    L0, nq, Hq, Hkv, D = args.kv_len, MEM_TOKENS + 1, 32, 8, 128
+    growth = (K + W) * nq + SEG_LEN + 64
+    cfg = synth.StepConfig("compress", B, Hq, Hkv, D, L0, L0, nq, 0, 5.0e5, 1024, headroom=growth, seed=0x5EED0004)
+    inp = synth.make_step_inputs(cfg, device=dev)
+    T = B * nq
+    # a1: UPL position IDs of the memory tokens and the PID of <o>, per sequence (host integer helpers)
+    pos = []
+    for b in range(B):
+        rho = inp.p0[b]
+        pos.append(np.concatenate([ms.memosight_upl_pids(rho, SEG_LEN, 3)[:MEM_TOKENS],
+                                   [ms.memosight_out_pid(rho, SEG_LEN)]]).astype(np.int32))
+    pos = torch.from_numpy(np.concatenate(pos)).to(dev)
+    q_work, ks_work = inp.q.clone(), inp.k_step.clone()
+    out = torch.empty((T, Hq, D), dtype=torch.bfloat16, device=dev)
+    max_kv = L0 + growth
+    wsb = ms.memosight_attn_workspace_bytes(B, Hq, Hkv, D, max_kv, nq)
+    ws = torch.empty(wsb, dtype=torch.uint8, device=dev)
+    stride = inp.n_slots * D
+    keep = torch.full((B,), nq, dtype=torch.int32, device=dev)
+    seg_len = torch.full((B,), SEG_LEN, dtype=torch.int32, device=dev)
+    seg_start = torch.empty(B, dtype=torch.int32, device=dev)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    for a_, b_ in evs:
+        a_.record()
+        b_.record()
+
+    def step(ev=None):
+        seg_start.copy_(inp.kv_len)                  # the finished step starts where the cache ended ...
+        inp.kv_len.add_(SEG_LEN)                     # ... and its 512 entries are in the cache
+        ms.memosight_rope_qk(q_work, ks_work, pos, T, Hq, Hkv, D, cfg.rope_base)
+        ms.memosight_attn_step(
+            batch=B, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, k_cache=inp.k_cache[0], v_cache=inp.v_cache[0],
+            kv_head_stride=stride, n_slots=inp.n_slots, kv_off=inp.kv_off, kv_len=inp.kv_len, max_kv_len=max_kv,
+            max_nq=nq, q_off=inp.q_off, n_cand=inp.n_cand, anchor=None, total_rows=T, sm_scale=0.0, q=q_work,
+            k_step=ks_work, v_step=inp.v_step, out=out, lse=None, workspace=ws, workspace_bytes=wsb,
+            ev_split_begin=None if ev is None else ev[0].cuda_event,
+            ev_split_end=None if ev is None else ev[1].cuda_event)
+        ms.memosight_kv_append(inp.k_cache[0], inp.v_cache[0], stride, B, Hkv, D, inp.kv_off, inp.kv_len, ks_work,
+                               inp.v_step, inp.q_off, inp.n_cand, keep, nq, 1)
+        ms.memosight_kv_compact(inp.k_cache, inp.v_cache, 1, Hkv * stride, stride, B, Hkv, D, inp.kv_off,
+                                inp.kv_len, seg_start, seg_len, None, 0, nq)
+
+    for _ in range(W):
+        step()
+    assert ms.memosight_attn_status(ws) == ms.MS_OK
+    sampler = ClockSampler(physical_gpu_index(int(os.environ.get("LOCAL_RANK", "0"))))
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    sampler.start()
+    e0.record()
+    for s_ in range(K):
+        step(evs[s_])
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.finish()
+    elapsed_ms = e0.elapsed_time(e1)
+    assert ms.memosight_attn_status(ws) == ms.MS_OK
+    assert inp.kv_len.cpu().tolist() == [L0 + (K + W) * nq] * B
+    attn_ms = float(np.mean([a_.elapsed_time(b_) for a_, b_ in evs]))
+    l_mid = L0 + SEG_LEN + (W + (K - 1) / 2.0) * nq
+    flops = 4.0 * B * Hq * D * nq * (l_mid + (nq + 1) / 2.0)       # visible keys: cache + causal half
+    sustained, burst, kind = peak_tensor()
+    achieved = flops / (attn_ms * 1e-3) / 1e12
+    line = {
+        "metric": "memory tokens/s (compression event: forward of 170 memory tokens + <o>, append, eviction of a "
+                  "512-token step; 8B shape)", "value": T * K / (elapsed_ms * 1e-3), "unit": "tokens/s", "n_gpus": 1,
+        "steps": K, "warmup": W, "ms_per_step": elapsed_ms / K, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"compression event, 8B-shape layer H_q={Hq} H_kv={Hkv} D={D}, batch {B}, cache "
+                               f"{L0} + a {SEG_LEN}-token step, block of {nq} causal tokens, 1 layer",
+                   "global_batch": B, "kv_len": L0, "block": nq,
+                   "l2": "K/V of one sequence-layer (69 MB) is re-read by the 6 row tiles of a KV head, mostly "
+                         "from L2; no flush"},
+        "roofline": {"bound": "tensor", "kernel": "attn_umma_big_kernel", "achieved": achieved, "peak": sustained,
+                     "peak_source": f"{kind} bf16 GEMM, sustained ({burst:.0f} burst)", "unit": "TFLOP/s",
+                     "frac": achieved / sustained, "avg_launch_ms": attn_ms, "algorithmic_flops_per_launch": flops,
+                     "traffic": None, "share_of_step_time": attn_ms * K / elapsed_ms},
+        "clocks": clocks, "gpu_launches": 8 * K,
+    }
+    print(json.dumps(line), flush=True)
 
 
 def run_e2e(ms, n_e2e, first, cfg, inp, acc, sched, seg_start, seg_len, ws, wsb, aws, awb, am, nm, nk, out, lse,
