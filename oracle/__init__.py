@@ -104,6 +104,13 @@ def monotone_pids(rho_first: int, n: int, c: int) -> np.ndarray:
     return out[:l].copy()
 
 
+def budget_pids(rho_first: int, n: int, l: int) -> np.ndarray:
+    out = np.empty(max(l, 1), dtype=np.int32)
+    r = int(lib().ms_oracle_budget_pids(C.c_int32(rho_first), C.c_int32(n), C.c_int32(l), _p(out, C.c_int32)))
+    _chk(min(r, 0), "budget_pids")
+    return out[:r].copy()
+
+
 def out_pid(rho_first: int, n: int) -> int:
     return int(lib().ms_oracle_out_pid(C.c_int32(rho_first), C.c_int32(n)))
 
@@ -184,6 +191,20 @@ def kv_compact(k_cache, v_cache, n_layers, layer_stride, kv_head_stride, H_kv, D
         _p(seg_len, C.c_int32), _p(src, C.c_int32), C.c_int32(idx_stride))
     _chk(rc, "kv_compact")
     return src
+
+
+def kv_gather(k_cache, v_cache, n_layers, layer_stride, kv_head_stride, H_kv, D, kv_off, kv_len, keep_idx, n_keep):
+    """In place on the uint16 arrays and on kv_len: new = old[keep_idx[b][:n_keep[b]]]."""
+    assert k_cache.dtype == np.uint16 and v_cache.dtype == np.uint16 and kv_len.dtype == np.int32
+    kv_off = np.ascontiguousarray(kv_off, dtype=np.int64)
+    keep_idx = np.ascontiguousarray(keep_idx, dtype=np.int32)
+    n_keep = np.ascontiguousarray(n_keep, dtype=np.int32)
+    B = kv_len.shape[0]
+    rc = lib().ms_oracle_kv_gather(
+        _p(k_cache, C.c_uint16), _p(v_cache, C.c_uint16), C.c_int32(n_layers), C.c_int64(layer_stride),
+        C.c_int64(kv_head_stride), C.c_int32(B), C.c_int32(H_kv), C.c_int32(D), _p(kv_off, C.c_int64),
+        _p(kv_len, C.c_int32), _p(keep_idx, C.c_int32), C.c_int32(keep_idx.shape[1]), _p(n_keep, C.c_int32))
+    _chk(rc, "kv_gather")
 
 
 def kv_append(k_cache, v_cache, kv_head_stride, H_kv, D, kv_off, kv_len, k_step, v_step, q_off,

@@ -130,6 +130,24 @@ int32_t ms_oracle_monotone_pids(int32_t rho_first, int32_t n, int32_t c,
   return l;
 }
 
+/* Ablation "w/o AMA" (App. B.3): a fixed budget of l memory tokens per step whatever its
+ * length n.  The paper does not say where they sit; reading taken here: the step is cut
+ * into l groups as evenly as possible, group g = offsets floor(g*n/l) .. floor((g+1)*n/l)-1,
+ * and memory token g takes its group's centre (floor), exactly as UPL does for its groups;
+ * a group left empty (n < l) takes the position it would start at, clamped into the step.
+ * Parity unpinned beyond the invariants.  Returns l, or a negative code. */
+int32_t ms_oracle_budget_pids(int32_t rho_first, int32_t n, int32_t l, int32_t* pid_out) {
+  if (n < 1 || l < 1) return MS_ORACLE_BAD_ARG;
+  for (int32_t g = 0; g < l; ++g) {
+    int64_t lo = (int64_t)g * n / l, hi = (int64_t)(g + 1) * n / l - 1;
+    if (hi < lo) hi = lo;                /* empty group */
+    if (lo > n - 1) lo = n - 1;
+    if (hi > n - 1) hi = n - 1;
+    pid_out[g] = rho_first + (int32_t)((lo + hi) / 2);
+  }
+  return l;
+}
+
 /* Output token <o> (Sec. 2.2 "Position ID Assignment"): PID of the step's last
  * reasoning token plus one, so reasoning and output tokens are consecutive. */
 int32_t ms_oracle_out_pid(int32_t rho_first, int32_t n) {
@@ -332,6 +350,36 @@ int32_t ms_oracle_kv_compact(uint16_t* k_cache, uint16_t* v_cache, int32_t n_lay
     kv_len[b] = newL;
     free(tmp);
     free(keep);
+  }
+  return MS_ORACLE_OK;
+}
+
+/* Eviction by an arbitrary keep list (the comparison systems of Sec. 4 -- heavy-hitter and
+ * separator-based eviction -- keep a different subset of the cache than MemoSight does, but
+ * the cache operation is the same): new = [old[keep[0]], old[keep[1]], ...], kv_len = n_keep.
+ * keep[b] must be strictly increasing and inside [0, L).  All layers, K and V, bits unchanged. */
+int32_t ms_oracle_kv_gather(uint16_t* k_cache, uint16_t* v_cache, int32_t n_layers,
+                            int64_t layer_stride, int64_t kv_head_stride, int32_t B,
+                            int32_t H_kv, int32_t D, const int64_t* kv_off, int32_t* kv_len,
+                            const int32_t* keep_idx, int32_t idx_stride, const int32_t* n_keep) {
+  for (int32_t b = 0; b < B; ++b) {
+    const int32_t L = kv_len[b], nk = n_keep[b];
+    const int32_t* keep = keep_idx + (int64_t)b * idx_stride;
+    if (nk < 0 || nk > L || nk > idx_stride) return MS_ORACLE_BAD_ARG;
+    for (int32_t j = 0; j < nk; ++j)
+      if (keep[j] < 0 || keep[j] >= L || (j > 0 && keep[j] <= keep[j - 1])) return MS_ORACLE_BAD_ARG;
+    uint16_t* tmp = (uint16_t*)malloc(sizeof(uint16_t) * (size_t)(nk + 1) * D);
+    for (int32_t layer = 0; layer < n_layers; ++layer)
+      for (int32_t kv = 0; kv < 2; ++kv)
+        for (int32_t h = 0; h < H_kv; ++h) {
+          uint16_t* base = (kv ? v_cache : k_cache) + layer * layer_stride +
+                           h * kv_head_stride + kv_off[b] * (int64_t)D;
+          for (int32_t j = 0; j < nk; ++j)
+            memcpy(tmp + (int64_t)j * D, base + (int64_t)keep[j] * D, sizeof(uint16_t) * D);
+          memcpy(base, tmp, sizeof(uint16_t) * (size_t)nk * D);
+        }
+    kv_len[b] = nk;
+    free(tmp);
   }
   return MS_ORACLE_OK;
 }

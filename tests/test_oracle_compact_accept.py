@@ -179,3 +179,48 @@ def test_argmax_ties_nan_inf_and_library():
     lg2 = np.concatenate([lg, np.full((40, 3), 1000.0, np.float32)], axis=1)
     am2, _ = oracle.accept(lg2, 257, [0, 40], [-1] * 40)
     assert np.array_equal(am2, am)
+
+
+def test_gather_by_keep_list_is_numpy_take_and_generalises_compaction():
+    n_layers, Hkv, D, slots = 2, 3, 4, 60
+    lens, offs = [10, 0, 25, 7], [0, 12, 13, 40]
+    rng = np.random.default_rng(3)
+    keeps = [sorted(rng.choice(L, size=rng.integers(0, L + 1), replace=False).tolist()) if L else [] for L in lens]
+    keeps[3] = list(range(7))                                   # keep everything: identity
+    idx = np.full((4, 32), -1, np.int32)
+    for b, kp in enumerate(keeps):
+        idx[b, :len(kp)] = kp
+    k, v = _cache(n_layers, Hkv, slots, D, 2)
+    k0, v0 = k.copy(), v.copy()
+    kv_len = np.array(lens, np.int32)
+    oracle.kv_gather(k, v, n_layers, Hkv * slots * D, slots * D, Hkv, D, np.array(offs), kv_len, idx,
+                     [len(kp) for kp in keeps])
+    for b, kp in enumerate(keeps):
+        assert kv_len[b] == len(kp)
+        for arr, arr0 in ((k, k0), (v, v0)):
+            want = np.take(arr0[:, :, offs[b]:offs[b] + lens[b]], np.array(kp, dtype=np.int64), axis=2)
+            assert np.array_equal(arr[:, :, offs[b]:offs[b] + len(kp)], want)
+    assert np.array_equal(k[:, :, 47:], k0[:, :, 47:])           # nobody's slots stay untouched
+    # the paper's eviction is the keep list "everything but the step": same result as kv_compact
+    k1, v1 = k0.copy(), v0.copy()
+    k2, v2 = k0.copy(), v0.copy()
+    len1, len2 = np.array(lens, np.int32), np.array(lens, np.int32)
+    seg_start, seg_len = [3, 0, 5, 2], [4, 0, 17, 3]
+    src = oracle.kv_compact(k1, v1, n_layers, Hkv * slots * D, slots * D, Hkv, D, np.array(offs), len1,
+                            seg_start, seg_len, idx_stride=32)
+    oracle.kv_gather(k2, v2, n_layers, Hkv * slots * D, slots * D, Hkv, D, np.array(offs), len2, src, len1)
+    assert np.array_equal(len1, len2)
+    for b in range(4):
+        sl = slice(offs[b], offs[b] + int(len1[b]))
+        assert np.array_equal(k1[:, :, sl], k2[:, :, sl]) and np.array_equal(v1[:, :, sl], v2[:, :, sl])
+
+
+def test_gather_rejects_bad_keep_lists():
+    k, v = _cache(1, 1, 10, 4, 5)
+    for bad in ([[2, 1]], [[0, 0]], [[9, 10]], [[-1, 3]]):
+        idx = np.array(bad, np.int32)
+        try:
+            oracle.kv_gather(k.copy(), v.copy(), 1, 40, 40, 1, 4, np.array([0]), np.array([10], np.int32), idx, [2])
+        except Exception:
+            continue
+        raise AssertionError(f"keep list {bad} was accepted")

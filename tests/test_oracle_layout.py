@@ -71,6 +71,22 @@ def test_monotone_pids_ablation():
     assert oracle.monotone_pids(10, 7, 3).tolist() == [17, 18, 19]
 
 
+def test_fixed_budget_pids_ablation():
+    # the "w/o AMA" variant: 9 memory tokens per step whatever its length (App. B.3)
+    for rho, n in ((0, 9), (100, 56), (7, 512), (3, 10), (50, 4), (0, 1)):
+        p = oracle.budget_pids(rho, n, 9)
+        assert len(p) == 9
+        assert np.all(np.diff(p) >= 0) and p[0] >= rho and p[-1] <= rho + n - 1    # ordered, inside the step
+        if n >= 9:
+            assert np.all(np.diff(p) >= 1)                                          # distinct when there is room
+            edges = [g * n // 9 for g in range(10)]
+            for g in range(9):
+                assert rho + edges[g] <= p[g] <= rho + edges[g + 1] - 1             # inside its own group
+    # with a budget that divides the step it is UPL with c = n / l
+    assert oracle.budget_pids(11, 45, 9).tolist() == oracle.upl_pids(11, 45, 5).tolist()
+    assert oracle.budget_pids(0, 9, 9).tolist() == list(range(9))
+
+
 def test_foresight_pid_paper_examples():
     for ex in GOLD["foresight_pid"]:
         got = oracle.step_pids(ex["p0"], ex["n_c"], ex["d"], ex.get("anchor")).tolist()
