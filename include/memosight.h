@@ -60,6 +60,9 @@ typedef void* memosight_stream_t; /* a cudaStream_t */
 #define MS_ROPE_NEOX 0u          /* pair (i, i + D/2): rotate-half, the default                  */
 #define MS_ROPE_INTERLEAVED 1u   /* pair (2i, 2i+1)                                              */
 #define MS_POS_HALF_UNITS 2u     /* pos_id counts half positions (exact UPL centres)             */
+/* Layout flag of memosight_upl_pids: the "w/o UPL" ablation of App. B.3 */
+#define MS_LAYOUT_MONOTONE 4u    /* memory tokens take fresh, monotonically increasing PIDs behind
+                                    the step (rho_first + n + g) instead of the group centres    */
 
 /* Library version (major*10000 + minor*100 + patch). */
 MS_API int32_t memosight_version(void);
@@ -78,10 +81,19 @@ MS_API int32_t memosight_ama(int32_t n, int32_t c);
  * and are cut into l = ceil(n/c) sequential groups of c (last may be shorter);
  * memory token g gets the centre PID of group g.  A half-integer centre (even
  * group size) is rounded down, or returned exactly in half positions when flags
- * has MS_POS_HALF_UNITS (value = 2*centre).  pid_out: host, capacity cap >= l.
+ * has MS_POS_HALF_UNITS (value = 2*centre).  With MS_LAYOUT_MONOTONE the groups are ignored
+ * and memory token g gets rho_first + n + g.  pid_out: host, capacity cap >= l.
  * Returns l, or a negative code (MS_ERR_INVALID_ARG also when cap < l). */
 MS_API int32_t memosight_upl_pids(int32_t rho_first, int32_t n, int32_t c, uint32_t flags,
                            int32_t* pid_out, int32_t cap);
+
+/* The "w/o AMA" ablation of App. B.3: a fixed budget of l memory tokens per step whatever its
+ * length n >= 1.  The step is cut into l groups as evenly as possible (group g = offsets
+ * floor(g*n/l) .. floor((g+1)*n/l)-1) and memory token g takes its group's centre, rounded
+ * down; a group left empty (n < l) takes the position it would start at, clamped into the
+ * step.  (The paper fixes only the budget, 9; the placement is this library's reading.)
+ * pid_out: host, capacity cap >= l.  Returns l or a negative code. */
+MS_API int32_t memosight_budget_pids(int32_t rho_first, int32_t n, int32_t l, int32_t* pid_out, int32_t cap);
 
 /* PID of the output token <o> that closes a step: the step's last PID plus one. */
 MS_API int32_t memosight_out_pid(int32_t rho_first, int32_t n);
@@ -206,6 +218,23 @@ MS_API int32_t memosight_kv_compact(void* k_cache, void* v_cache, int32_t n_laye
                              int32_t head_dim, const int64_t* kv_off, int32_t* kv_len,
                              const int32_t* seg_start, const int32_t* seg_len, int32_t* src_idx,
                              int32_t idx_stride, int32_t max_tail, memosight_stream_t stream);
+
+/* Eviction by an arbitrary keep list, in place, every layer, K and V:
+ *     new = [old[keep_idx[b][0]], old[keep_idx[b][1]], ...],  kv_len[b] = n_keep[b].
+ * MemoSight's own eviction is the special case "everything but the finished step"
+ * (memosight_kv_compact, which also emits that list); the eviction policies the paper compares
+ * with (heavy-hitter and separator-based, Sec. 4) keep other subsets through the same operation.
+ *   keep_idx  device int32 [B][idx_stride]: strictly increasing old indices, all < kv_len[b]
+ *   n_keep    device int32 [B], 0 <= n_keep[b] <= min(kv_len[b], idx_stride)
+ *   max_keep  host upper bound of n_keep[]
+ * A row whose list is not strictly increasing or leaves [0, kv_len) is undefined behaviour
+ * within the sequence's own slots (nothing outside them is read or written).  Other arguments
+ * as for memosight_kv_compact. */
+MS_API int32_t memosight_kv_gather(void* k_cache, void* v_cache, int32_t n_layers, int64_t layer_stride,
+                            int64_t kv_head_stride, int32_t batch, int32_t n_kv_heads, int32_t head_dim,
+                            const int64_t* kv_off, int32_t* kv_len, const int32_t* keep_idx,
+                            int32_t idx_stride, const int32_t* n_keep, int32_t max_keep,
+                            memosight_stream_t stream);
 
 /* Appends the accepted candidates of each block to one layer's cache: the first
  * n_keep[b] rows of block b in k_step/v_step go to slots kv_len[b] .. of sequence

@@ -35,6 +35,7 @@ MS_ATTN_PATH_TCGEN05_KEYS = 4
 MS_ROPE_NEOX = 0
 MS_ROPE_INTERLEAVED = 1
 MS_POS_HALF_UNITS = 2
+MS_LAYOUT_MONOTONE = 4
 
 
 class MemosightError(RuntimeError):
@@ -119,6 +120,12 @@ def lib() -> C.CDLL:
         L.memosight_kv_compact.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int64, C.c_int64, C.c_int32,
                                            C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
                                            C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p]
+        L.memosight_budget_pids.restype = C.c_int32
+        L.memosight_budget_pids.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_int32]
+        L.memosight_kv_gather.restype = C.c_int32
+        L.memosight_kv_gather.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int64, C.c_int64, C.c_int32,
+                                          C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
+                                          C.c_void_p, C.c_int32, C.c_void_p]
         L.memosight_kv_append.restype = C.c_int32
         L.memosight_kv_append.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_int32,
                                           C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
@@ -183,6 +190,14 @@ def memosight_upl_pids(rho_first: int, n: int, c: int, flags: int = 0) -> np.nda
     r = int(lib().memosight_upl_pids(rho_first, n, c, flags, out.ctypes.data, out.size))
     if r < 0:
         raise MemosightError(r, "memosight_upl_pids")
+    return out[:r].copy()
+
+
+def memosight_budget_pids(rho_first: int, n: int, l: int) -> np.ndarray:
+    out = np.empty(max(l, 1), dtype=np.int32)
+    r = int(lib().memosight_budget_pids(rho_first, n, l, out.ctypes.data, out.size))
+    if r < 0:
+        raise MemosightError(r, "memosight_budget_pids")
     return out[:r].copy()
 
 
@@ -266,6 +281,14 @@ def memosight_kv_compact(k_cache, v_cache, n_layers, layer_stride, kv_head_strid
                                           batch, n_kv_heads, head_dim, _ptr(kv_off), _ptr(kv_len),
                                           _ptr(seg_start), _ptr(seg_len), _ptr(src_idx), idx_stride, max_tail,
                                           _stream(stream))), "memosight_kv_compact")
+
+
+def memosight_kv_gather(k_cache, v_cache, n_layers, layer_stride, kv_head_stride, batch, n_kv_heads, head_dim,
+                        kv_off, kv_len, keep_idx, idx_stride, n_keep, max_keep, stream=None) -> None:
+    _check(int(lib().memosight_kv_gather(_ptr(k_cache), _ptr(v_cache), n_layers, layer_stride, kv_head_stride,
+                                         batch, n_kv_heads, head_dim, _ptr(kv_off), _ptr(kv_len), _ptr(keep_idx),
+                                         idx_stride, _ptr(n_keep), max_keep, _stream(stream))),
+           "memosight_kv_gather")
 
 
 def memosight_kv_append(k_cache, v_cache, kv_head_stride, batch, n_kv_heads, head_dim, kv_off, kv_len, k_step,

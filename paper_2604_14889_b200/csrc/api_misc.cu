@@ -53,12 +53,32 @@ int32_t memosight_upl_pids(int32_t rho_first, int32_t n, int32_t c, uint32_t fla
   const int32_t l = memosight_ama(n, c);
   if (l < 0) return l;
   if (l > 0 && (pid_out == nullptr || cap < l)) return MS_ERR_INVALID_ARG;
+  if (flags & ~(MS_POS_HALF_UNITS | MS_LAYOUT_MONOTONE)) return MS_ERR_INVALID_ARG;
+  if (flags & MS_LAYOUT_MONOTONE) {   // "w/o UPL": fresh PIDs behind the step, one per memory token
+    const int32_t unit = (flags & MS_POS_HALF_UNITS) ? 2 : 1;
+    for (int32_t g = 0; g < l; ++g) pid_out[g] = unit * (rho_first + n + g);
+    return l;
+  }
   for (int32_t g = 0; g < l; ++g) {
     const int64_t first = static_cast<int64_t>(g) * c;               // offsets inside the step
     const int64_t last = (first + c < n ? first + c : n) - 1;
     const int64_t twice_centre = 2 * static_cast<int64_t>(rho_first) + first + last;
     pid_out[g] = static_cast<int32_t>((flags & MS_POS_HALF_UNITS) ? twice_centre
                                                                  : (twice_centre >> 1));
+  }
+  return l;
+}
+
+// Fixed budget of l memory tokens ("w/o AMA"): l groups cut as evenly as possible.
+int32_t memosight_budget_pids(int32_t rho_first, int32_t n, int32_t l, int32_t* pid_out, int32_t cap) {
+  if (n < 1 || l < 1 || pid_out == nullptr || cap < l) return MS_ERR_INVALID_ARG;
+  for (int32_t g = 0; g < l; ++g) {
+    int64_t first = static_cast<int64_t>(g) * n / l;
+    int64_t last = static_cast<int64_t>(g + 1) * n / l - 1;
+    if (last < first) last = first;               // empty group: where it would start
+    if (first > n - 1) first = n - 1;
+    if (last > n - 1) last = n - 1;
+    pid_out[g] = rho_first + static_cast<int32_t>((first + last) >> 1);
   }
   return l;
 }

@@ -496,7 +496,6 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
       // p = 2^x as bf16 into this row of the P tile (half g = this group's 64 keys)
       {
         const uint32_t p_row = sb + kBOffP + pb * kBPBytes + wg * kBHalf + r * 128;
-#pragma unroll
         float ls[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int c = 0; c < 8; ++c) {

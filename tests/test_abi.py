@@ -54,7 +54,7 @@ def test_host_side_validation_codes():
     assert L.memosight_kv_append(None, None, 0, 2, 1, 64, None, None, None, None, None, None, None, 4, 1, None) \
         == ms.MS_ERR_INVALID_ARG
     assert L.memosight_attn_workspace_bytes(1, 5, 2, 64, 10, 4) == 0          # H_q % H_kv != 0
-    assert L.memosight_attn_workspace_bytes(1, 4, 2, 64, 10, 17) == 0         # block too large
+    assert L.memosight_attn_workspace_bytes(1, 4, 2, 64, 10, 257) == 0        # block too large
     assert L.memosight_attn_workspace_bytes(1, 4, 2, 64, 10, 4) > 256
 
     def params(**kw):
@@ -67,7 +67,7 @@ def test_host_side_validation_codes():
         return p
     assert L.memosight_attn_step(C.byref(params(n_q_heads=5)), None) == ms.MS_ERR_INVALID_ARG
     assert L.memosight_attn_step(C.byref(params(head_dim=48)), None) == ms.MS_ERR_UNSUPPORTED_SHAPE
-    assert L.memosight_attn_step(C.byref(params(max_nq=17)), None) == ms.MS_ERR_UNSUPPORTED_SHAPE
+    assert L.memosight_attn_step(C.byref(params(max_nq=257)), None) == ms.MS_ERR_UNSUPPORTED_SHAPE
     assert L.memosight_attn_step(C.byref(params()), None) == ms.MS_ERR_INVALID_ARG       # null pointers
     fake = 0x1000
     full = dict(k_cache=fake, v_cache=fake, kv_off=fake, kv_len=fake, q_off=fake, n_cand=fake, q=fake,
@@ -88,8 +88,17 @@ def test_layout_helpers_agree_with_oracle():
                 assert ms.memosight_upl_pids(rho, n, c, ms.MS_POS_HALF_UNITS).tolist() == \
                     oracle.upl_pids(rho, n, c, half_units=True).tolist()
                 assert ms.memosight_out_pid(rho, n) == oracle.out_pid(rho, n)
+                # ablation layouts (App. B.3): monotone PIDs (w/o UPL), fixed budget (w/o AMA)
+                assert ms.memosight_upl_pids(rho, n, c, ms.MS_LAYOUT_MONOTONE).tolist() == \
+                    oracle.monotone_pids(rho, n, c).tolist()
+                if n >= 1:
+                    assert ms.memosight_budget_pids(rho, n, c).tolist() == oracle.budget_pids(rho, n, c).tolist()
     with pytest.raises(ms.MemosightError):
         ms.memosight_ama(3, 0)
+    with pytest.raises(ms.MemosightError):
+        ms.memosight_budget_pids(0, 0, 9)
+    with pytest.raises(ms.MemosightError):
+        ms.memosight_upl_pids(0, 5, 2, 8)
     for p0 in (0, 9, 50000):
         for n_c in range(0, 6):
             for d in range(0, 6):

@@ -319,3 +319,63 @@ def test_generator_is_identical_on_cpu_and_gpu():
     c = synth.normal_f32(100000, 3, synth.STREAM_LOGITS, 2.0, device="cpu", offset=999)
     d = synth.normal_f32(100000, 3, synth.STREAM_LOGITS, 2.0, device=DEV, offset=999)
     assert torch.equal(c, d.cpu())
+
+
+# --------------------------------------------------------------------------- eviction by keep list
+
+def _gather_both(inp, keeps, idx_stride):
+    c = inp.cfg
+    B = c.batch
+    idx = np.full((B, idx_stride), -1, np.int32)
+    for b, kp in enumerate(keeps):
+        idx[b, :len(kp)] = kp
+    n_keep = np.array([len(kp) for kp in keeps], np.int32)
+    kb, vb = bits(inp.k_cache), bits(inp.v_cache)
+    kv_len = inp.kv_len.cpu().numpy().copy()
+    layer_stride = c.n_kv_heads * inp.n_slots * c.head_dim
+    oracle.kv_gather(kb, vb, c.n_layers, layer_stride, inp.n_slots * c.head_dim, c.n_kv_heads, c.head_dim,
+                     inp.kv_off.cpu().numpy(), kv_len, idx, n_keep)
+    gk, gv = inp.k_cache.to(DEV).clone(), inp.v_cache.to(DEV).clone()
+    g_len = inp.kv_len.to(DEV).clone()
+    ms.memosight_kv_gather(gk, gv, c.n_layers, layer_stride, inp.n_slots * c.head_dim, B, c.n_kv_heads,
+                           c.head_dim, inp.kv_off.to(DEV), g_len, torch.from_numpy(idx).to(DEV), idx_stride,
+                           torch.from_numpy(n_keep).to(DEV), int(n_keep.max()))
+    torch.cuda.synchronize()
+    assert np.array_equal(g_len.cpu().numpy(), kv_len)
+    for b in range(B):
+        sl = slice(inp.offs[b], inp.offs[b] + int(kv_len[b]))
+        assert np.array_equal(bits(gk[:, :, sl]), kb[:, :, sl]) and np.array_equal(bits(gv[:, :, sl]), vb[:, :, sl])
+    # slots of other sequences' slack and everything beyond the old lengths are never written
+    for b in range(B):
+        sl = slice(inp.offs[b] + inp.lens[b], inp.offs[b] + inp.lens[b] + c.headroom)
+        assert np.array_equal(bits(gk[:, :, sl]), bits(inp.k_cache[:, :, sl]))
+
+
+def test_gather_keep_lists_of_other_eviction_policies():
+    cfg = synth.StepConfig("g", 6, 8, 4, 128, 300, 2600, 3, 3, 1e4, 100, n_layers=2, seed=91, headroom=32)
+    inp = synth.make_step_inputs(cfg)
+    rng = np.random.default_rng(4)
+    keeps = []
+    for b, L in enumerate(inp.lens):
+        if b == 0:      # heavy-hitter style: a recent window plus scattered older entries
+            old = sorted(rng.choice(L - 256, size=128, replace=False).tolist())
+            keeps.append(old + list(range(L - 256, L)))
+        elif b == 1:    # separator style: initial tokens, every 17th entry, the neighbourhood
+            keeps.append(sorted(set(range(4)) | set(range(0, L, 17)) | set(range(L - 64, L))))
+        elif b == 2:    # keep everything
+            keeps.append(list(range(L)))
+        elif b == 3:    # keep nothing
+            keeps.append([])
+        elif b == 4:    # the method's own eviction: everything but one step
+            keeps.append(list(range(0, 50)) + list(range(50 + 200, L)))
+        else:           # only the last entry
+            keeps.append([L - 1])
+    _gather_both(inp, keeps, 2700)
+
+
+def test_gather_random_lists_and_head_dim_64():
+    cfg = synth.StepConfig("g64", 9, 4, 2, 64, 1, 700, 3, 3, 1e4, 100, n_layers=3, seed=92, headroom=16)
+    inp = synth.make_step_inputs(cfg)
+    rng = np.random.default_rng(5)
+    keeps = [sorted(rng.choice(L, size=int(rng.integers(0, L + 1)), replace=False).tolist()) for L in inp.lens]
+    _gather_both(inp, keeps, 704)
