@@ -302,6 +302,76 @@ MS_API int32_t memosight_accept_static(const float* logits, int64_t ld_v, int32_
                                        const int32_t* draft, int32_t* argmax_out, int32_t* n_match,
                                        int32_t* n_keep, memosight_stream_t stream);
 
+/* ---- Bookkeeping of the iterative inference loop (App. A, Algorithm 1) --------------------- */
+
+/* Per-sequence decoding state, all of it in device memory owned by the caller.  The calls
+ * below only read and update it with kernels on `stream`; nothing is copied to the host.
+ * A sequence starts with cand[b][0] = its first token (verified by the prefill), n_cand = 1,
+ * pos_next = that token's position ID, seg_start = kv_len (the reasoning step starts behind
+ * the prompt), seg_n = 0, seg_pid0 = pos_next, flags = 0, n_out = 0. */
+typedef struct memosight_decode_state {
+  uint32_t struct_size;   /* sizeof(memosight_decode_state)                                     */
+  int32_t batch;          /* B                                                                   */
+  int32_t d;              /* foresight tokens per block, 0..7 (a block has at most 2d+1 rows)    */
+  int32_t c;              /* compression ratio of AMA: l = ceil(n / c)                           */
+  int32_t max_out;        /* capacity of out_tok per sequence; reaching it ends the sequence     */
+  int32_t max_mem;        /* upper bound of l, 1..255 (longer steps get max_mem memory tokens)   */
+  int32_t tok_foresight, tok_memory, tok_output;   /* ids of <f>, <m>, <o>                       */
+  int32_t tok_delim, tok_eos;                      /* step delimiter (<e>) and end of sequence   */
+  int32_t* kv_len;        /* [B] cache lengths: the array the cache calls update                 */
+  int32_t* pos_next;      /* [B] position ID of cand[b][0]                                       */
+  int32_t* seg_start;     /* [B] cache index of the current reasoning step's first entry         */
+  int32_t* seg_n;         /* [B] entries of the current step in the cache so far                 */
+  int32_t* seg_pid0;      /* [B] position ID of the current step's first token                   */
+  int32_t* cand;          /* [B][d+1] pending candidates: c_0 verified, the others are drafts    */
+  int32_t* n_cand;        /* [B] 1..d+1                                                          */
+  int32_t* flags;         /* [B] bit 0: finished; bit 1: step ended, compression pending         */
+  int32_t* out_tok;       /* [B][max_out] the permanent tokens in order                          */
+  int32_t* n_out;         /* [B] tokens made permanent so far (may exceed max_out by the last block) */
+} memosight_decode_state;
+
+/* Device scratch needed by the two plan calls. */
+MS_API size_t memosight_decode_scratch_bytes(int32_t batch);
+
+/* Builds the Predict+Verify block of every live sequence (not finished, no compression
+ * pending): rows c_0..c_{n-1} then d foresight tokens (Sec. 2.1.1).
+ *   q_off [B+1], n_cand_blk [B]   as memosight_attn_params wants them (empty block = skipped)
+ *   row_tok [T], pos_id [T]       token id to embed and position ID of every row
+ *   draft [T]                     what memosight_accept has to find: c_{i+1}, or -1
+ *   summary [4]                   {rows in total, live sequences, sequences waiting for
+ *                                 compression, 0}: the one thing a host loop reads back
+ * Arrays are device memory sized for T = B * (2d+1) rows. */
+MS_API int32_t memosight_decode_plan(const memosight_decode_state* state, int32_t* q_off, int32_t* n_cand_blk,
+                              int32_t* row_tok, int32_t* pos_id, int32_t* draft, int32_t* summary,
+                              void* scratch, memosight_stream_t stream);
+
+/* Applies the greedy verification (argmax, n_match from memosight_accept on this block):
+ * c_0..c_m become permanent (m = matching prefix), cut behind the first delimiter or
+ * end-of-sequence token among them (which sets the flag) or at the output budget; n_keep[b]
+ * says how many, for memosight_kv_append.  The prediction behind the last permanent token is
+ * the next c_0; if every candidate was accepted and the step goes on, the d foresight
+ * predictions are the next drafts, otherwise they are dropped (they were conditioned on all
+ * candidates).  Does not touch kv_len: the append does. */
+MS_API int32_t memosight_decode_commit(const memosight_decode_state* state, const int32_t* q_off,
+                                const int32_t* argmax, const int32_t* n_match, int32_t* n_keep,
+                                memosight_stream_t stream);
+
+/* Builds the compression block of every sequence whose step has ended (Sec. 2.1.2):
+ * l = ceil(seg_n / c) memory tokens at the centres of their groups (UPL, rounded down) and <o> at
+ * the step's last position + 1, all candidates (causal).  n_keep [B] = l + 1 for the append;
+ * seg_start / seg_len [B] are the eviction request for memosight_kv_compact (0 = skip).
+ * Arrays sized for T = B * (max_mem + 1) rows.  summary as above. */
+MS_API int32_t memosight_decode_plan_compress(const memosight_decode_state* state, int32_t* q_off,
+                                       int32_t* n_cand_blk, int32_t* row_tok, int32_t* pos_id,
+                                       int32_t* n_keep, int32_t* seg_start, int32_t* seg_len,
+                                       int32_t* summary, void* scratch, memosight_stream_t stream);
+
+/* After the compression block was forwarded, appended and the step evicted (kv_len final):
+ * the next step starts behind <o>, whose prediction (argmax of the block's last row) is its
+ * first token; clears the pending flag. */
+MS_API int32_t memosight_decode_commit_compress(const memosight_decode_state* state, const int32_t* q_off,
+                                         const int32_t* argmax, memosight_stream_t stream);
+
 /* ---- One whole step with the step's inputs and results in host memory -------------------- */
 
 /* The KV cache is device-resident state (it is what the method keeps compacted);

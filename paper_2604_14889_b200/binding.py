@@ -82,6 +82,19 @@ class StepHostParams(C.Structure):
     ]
 
 
+class DecodeState(C.Structure):
+    """Mirror of ``memosight_decode_state`` (include/memosight.h)."""
+    _fields_ = [
+        ("struct_size", C.c_uint32), ("batch", C.c_int32), ("d", C.c_int32), ("c", C.c_int32),
+        ("max_out", C.c_int32), ("max_mem", C.c_int32),
+        ("tok_foresight", C.c_int32), ("tok_memory", C.c_int32), ("tok_output", C.c_int32),
+        ("tok_delim", C.c_int32), ("tok_eos", C.c_int32),
+        ("kv_len", C.c_void_p), ("pos_next", C.c_void_p), ("seg_start", C.c_void_p), ("seg_n", C.c_void_p),
+        ("seg_pid0", C.c_void_p), ("cand", C.c_void_p), ("n_cand", C.c_void_p), ("flags", C.c_void_p),
+        ("out_tok", C.c_void_p), ("n_out", C.c_void_p),
+    ]
+
+
 _lib: Optional[C.CDLL] = None
 
 
@@ -126,6 +139,16 @@ def lib() -> C.CDLL:
         L.memosight_kv_gather.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int64, C.c_int64, C.c_int32,
                                           C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
                                           C.c_void_p, C.c_int32, C.c_void_p]
+        L.memosight_decode_scratch_bytes.restype = C.c_size_t
+        L.memosight_decode_scratch_bytes.argtypes = [C.c_int32]
+        L.memosight_decode_plan.restype = C.c_int32
+        L.memosight_decode_plan.argtypes = [C.POINTER(DecodeState)] + [C.c_void_p] * 8
+        L.memosight_decode_commit.restype = C.c_int32
+        L.memosight_decode_commit.argtypes = [C.POINTER(DecodeState)] + [C.c_void_p] * 5
+        L.memosight_decode_plan_compress.restype = C.c_int32
+        L.memosight_decode_plan_compress.argtypes = [C.POINTER(DecodeState)] + [C.c_void_p] * 10
+        L.memosight_decode_commit_compress.restype = C.c_int32
+        L.memosight_decode_commit_compress.argtypes = [C.POINTER(DecodeState)] + [C.c_void_p] * 3
         L.memosight_kv_append.restype = C.c_int32
         L.memosight_kv_append.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_int32,
                                           C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
@@ -281,6 +304,49 @@ def memosight_kv_compact(k_cache, v_cache, n_layers, layer_stride, kv_head_strid
                                           batch, n_kv_heads, head_dim, _ptr(kv_off), _ptr(kv_len),
                                           _ptr(seg_start), _ptr(seg_len), _ptr(src_idx), idx_stride, max_tail,
                                           _stream(stream))), "memosight_kv_compact")
+
+
+def decode_state(batch, d, c, max_out, max_mem, tok_foresight, tok_memory, tok_output, tok_delim, tok_eos,
+                 kv_len, pos_next, seg_start, seg_n, seg_pid0, cand, n_cand, flags, out_tok, n_out) -> DecodeState:
+    """Fills a ``memosight_decode_state`` from tensors / addresses."""
+    st = DecodeState()
+    st.struct_size = C.sizeof(DecodeState)
+    st.batch, st.d, st.c, st.max_out, st.max_mem = batch, d, c, max_out, max_mem
+    st.tok_foresight, st.tok_memory, st.tok_output = tok_foresight, tok_memory, tok_output
+    st.tok_delim, st.tok_eos = tok_delim, tok_eos
+    for name, t in (("kv_len", kv_len), ("pos_next", pos_next), ("seg_start", seg_start), ("seg_n", seg_n),
+                    ("seg_pid0", seg_pid0), ("cand", cand), ("n_cand", n_cand), ("flags", flags),
+                    ("out_tok", out_tok), ("n_out", n_out)):
+        setattr(st, name, _ptr(t))
+    return st
+
+
+def memosight_decode_scratch_bytes(batch: int) -> int:
+    return int(lib().memosight_decode_scratch_bytes(batch))
+
+
+def memosight_decode_plan(state, q_off, n_cand_blk, row_tok, pos_id, draft, summary, scratch, stream=None) -> None:
+    _check(int(lib().memosight_decode_plan(C.byref(state), _ptr(q_off), _ptr(n_cand_blk), _ptr(row_tok),
+                                           _ptr(pos_id), _ptr(draft), _ptr(summary), _ptr(scratch),
+                                           _stream(stream))), "memosight_decode_plan")
+
+
+def memosight_decode_commit(state, q_off, argmax, n_match, n_keep, stream=None) -> None:
+    _check(int(lib().memosight_decode_commit(C.byref(state), _ptr(q_off), _ptr(argmax), _ptr(n_match),
+                                             _ptr(n_keep), _stream(stream))), "memosight_decode_commit")
+
+
+def memosight_decode_plan_compress(state, q_off, n_cand_blk, row_tok, pos_id, n_keep, seg_start, seg_len, summary,
+                                   scratch, stream=None) -> None:
+    _check(int(lib().memosight_decode_plan_compress(C.byref(state), _ptr(q_off), _ptr(n_cand_blk), _ptr(row_tok),
+                                                    _ptr(pos_id), _ptr(n_keep), _ptr(seg_start), _ptr(seg_len),
+                                                    _ptr(summary), _ptr(scratch), _stream(stream))),
+           "memosight_decode_plan_compress")
+
+
+def memosight_decode_commit_compress(state, q_off, argmax, stream=None) -> None:
+    _check(int(lib().memosight_decode_commit_compress(C.byref(state), _ptr(q_off), _ptr(argmax),
+                                                      _stream(stream))), "memosight_decode_commit_compress")
 
 
 def memosight_kv_gather(k_cache, v_cache, n_layers, layer_stride, kv_head_stride, batch, n_kv_heads, head_dim,

@@ -290,3 +290,76 @@ def make_accept_inputs(cfg: StepConfig, device="cpu", plant: bool = True, pad: i
         logits=logits, ld_v=ld_v,
         row_off=torch.arange(0, T + 1, nq, dtype=torch.int32, device=dev),
         draft=torch.tensor(draft, dtype=torch.int32, device=dev), target=target)
+
+
+# --------------------------------------------------------------------------- #
+# A toy "model" for driving the inference loop                                 #
+# --------------------------------------------------------------------------- #
+
+STREAM_TOY_TOKEN, STREAM_TOY_HIT, STREAM_TOY_DELIM, STREAM_TOY_ROW = 20, 21, 22, 23
+
+
+@dataclasses.dataclass(frozen=True)
+class ToyModel:
+    """Stands in for the language model when the decoding loop is exercised: there are no
+    weights in this repository.  Every sequence has a fixed "true" continuation indexed by
+    position ID; a regular row (a candidate, or <o>) predicts the true token of the next
+    position; a foresight row predicts it only with probability `hit_pct` % (decided by a hash
+    of sequence and position), otherwise a wrong token -- which is what makes drafts fail.  The
+    q/k/v rows handed to the attention are pseudo-random functions of (sequence, token,
+    position, layer).  Holds no arithmetic of the method: it only produces its inputs."""
+    vocab: int = 1000           # regular tokens are 0 .. vocab-6; the specials sit above
+    hit_pct: int = 60
+    step_len: int = 23          # a delimiter roughly every step_len positions
+    eos_after: int = 400        # positions (from the sequence's first) after which <eos> comes
+    seed: int = 0x70F0
+
+    @property
+    def tok_f(self): return self.vocab - 5
+    @property
+    def tok_m(self): return self.vocab - 4
+    @property
+    def tok_o(self): return self.vocab - 3
+    @property
+    def tok_delim(self): return self.vocab - 2
+    @property
+    def tok_eos(self): return self.vocab - 1
+
+    def truth(self, b: int, pid: int, pid0: int) -> int:
+        """True token of sequence b at position pid (pid0 = the sequence's first position)."""
+        if pid - pid0 >= self.eos_after:
+            return self.tok_eos
+        if hash_scalar(b * 1000003 + pid, self.seed, STREAM_TOY_DELIM) % self.step_len == 0:
+            return self.tok_delim
+        return hash_scalar(b * 1000003 + pid, self.seed, STREAM_TOY_TOKEN) % (self.vocab - 5)
+
+    def predict(self, b: int, tok: int, pid: int, pid0: int) -> int:
+        """Token the model's head puts first on a row holding `tok` at position `pid`."""
+        t = self.truth(b, pid + 1, pid0)
+        if tok == self.tok_f and hash_scalar(b * 1000003 + pid, self.seed, STREAM_TOY_HIT) % 100 >= self.hit_pct:
+            return (t + 1) % (self.vocab - 5)
+        if tok == self.tok_m:
+            return hash_scalar(pid, self.seed, STREAM_TOY_TOKEN) % (self.vocab - 5)
+        return t
+
+    def logits(self, seq_of_row, row_tok, pos_id, pid0) -> torch.Tensor:
+        """fp32 [T][vocab]: small seeded noise with the predicted token planted 40 above it."""
+        T = len(row_tok)
+        lg = normal_f32(T * self.vocab, self.seed, STREAM_LOGITS, 2.0).view(T, self.vocab).clone()
+        for r in range(T):
+            lg[r, self.predict(int(seq_of_row[r]), int(row_tok[r]), int(pos_id[r]), pid0[int(seq_of_row[r])])] += 40.0
+        return lg
+
+    def qkv(self, seq_of_row, row_tok, pos_id, layer: int, Hq: int, Hkv: int, D: int):
+        """bf16 q [T][Hq][D], k, v [T][Hkv][D] of one layer: each row is its own seeded draw."""
+        T = len(row_tok)
+        q = torch.empty((T, Hq, D), dtype=torch.bfloat16)
+        k = torch.empty((T, Hkv, D), dtype=torch.bfloat16)
+        v = torch.empty((T, Hkv, D), dtype=torch.bfloat16)
+        for r in range(T):
+            key = hash_scalar((int(seq_of_row[r]) * 4099 + int(row_tok[r])) * 65537 + int(pos_id[r]) * 7 + layer,
+                              self.seed, STREAM_TOY_ROW) % (1 << 40)
+            q[r] = normal_bf16(Hq * D, self.seed, STREAM_Q, offset=key).view(Hq, D)
+            k[r] = normal_bf16(Hkv * D, self.seed, STREAM_KSTEP, offset=key).view(Hkv, D)
+            v[r] = normal_bf16(Hkv * D, self.seed, STREAM_VSTEP, offset=key).view(Hkv, D)
+        return q, k, v
