@@ -143,7 +143,7 @@ typedef struct memosight_attn_params {
   const int64_t* kv_off;     /* device [B]: first slot of sequence b                           */
   const int32_t* kv_len;     /* device [B]: valid entries L_b (kv_off[b]+L_b <= n_slots)       */
   int32_t max_kv_len;        /* host upper bound of kv_len[]                                   */
-  int32_t max_nq;            /* host upper bound of the block sizes, 1..256                    */
+  int32_t max_nq;            /* host upper bound of the block sizes, 1..32768                  */
   const int32_t* q_off;      /* device [B+1]: rows of block b are q_off[b] .. q_off[b+1]-1     */
   const int32_t* n_cand;     /* device [B]: candidates in block b (the block's first rows)     */
   const int32_t* anchor;     /* device [T] or NULL; read only for foresight rows               */
@@ -166,11 +166,13 @@ MS_API size_t memosight_attn_workspace_bytes(int32_t batch, int32_t n_q_heads, i
                                       int32_t head_dim, int32_t max_kv_len, int32_t max_nq);
 
 /* Queues the attention of one layer (split-KV pass + log-sum-exp merge).
- * Limits: n_q_heads/n_kv_heads <= 16; max_nq <= 256; batch <= 8192 per call.
+ * Limits: n_q_heads/n_kv_heads <= 16; max_nq <= 32768; batch <= 8192 per call.
  * Step blocks (max_nq <= 16) with max_nq * (H_q/H_kv) <= 128 and D in {64,128} take a
  * tensor-core kernel (see memosight_attn_set_path).  Larger blocks -- the compression pass
  * forwards the ceil(n/c) memory tokens and <o> of a finished step as one causal block
- * (Sec. 2.1.2, Algorithm 1) -- take the large-block tcgen05 kernel when D is 128.  Anything
+ * (Sec. 2.1.2, Algorithm 1), and the prefill of a prompt is one causal block against an empty
+ * or partly filled cache (Algorithm 1, Prefill) -- take the large-block tcgen05 kernel when D
+ * is 128.  Anything
  * else inside the limits takes the slower general kernel.  Pass the max_nq the workspace was
  * sized for: the workspace of a large-block call is bigger.
  * The workspace may be reused by the next call on the same stream; two calls

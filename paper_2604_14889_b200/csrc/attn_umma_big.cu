@@ -1,10 +1,11 @@
-// tcgen05 attention for large blocks (17..256 new tokens per sequence), head_dim 128.
+// tcgen05 attention for large blocks (17..32768 new tokens per sequence), head_dim 128.
 //
 // MemoSight's compression pass (paper Sec. 2.1.2; Algorithm 1, the forward over the l memory
 // tokens and <o> appended behind a finished reasoning step) is the same masked attention as
 // a Predict+Verify step -- whole compacted cache visible, the block's own tokens causal -- but
 // with up to ceil(512/3)+1 = 172 tokens in the block, i.e. several hundred packed rows per KV
-// head.  The block is cut into row tiles of floor(128/G) tokens (<= 128 packed rows); a work
+// head.  The prefill of a prompt (Algorithm 1, Prefill) is the same call with a longer block and
+// an empty cache.  The block is cut into row tiles of floor(128/G) tokens (<= 128 packed rows); a work
 // unit is (sequence, KV head, row tile) and streams the whole cache plus the step-local key
 // tiles up to its own last token (later keys are invisible to all of its rows).
 //

@@ -35,7 +35,7 @@ int32_t sm_count();
 inline cudaStream_t as_stream(memosight_stream_t s) { return reinterpret_cast<cudaStream_t>(s); }
 
 constexpr int kMaxNq = 16;        // largest step block of the Predict+Verify kernels
-constexpr int kMaxNqBig = 256;    // largest block of the large-block (compression pass) kernel
+constexpr int kMaxNqBig = 32768;  // largest block of the large-block kernel (compression pass, prefill)
 constexpr int kMaxGroup = 16;     // largest H_q / H_kv
 constexpr int kMaxBatch = 8192;   // sequences per attention launch
 

@@ -54,7 +54,7 @@ def test_host_side_validation_codes():
     assert L.memosight_kv_append(None, None, 0, 2, 1, 64, None, None, None, None, None, None, None, 4, 1, None) \
         == ms.MS_ERR_INVALID_ARG
     assert L.memosight_attn_workspace_bytes(1, 5, 2, 64, 10, 4) == 0          # H_q % H_kv != 0
-    assert L.memosight_attn_workspace_bytes(1, 4, 2, 64, 10, 257) == 0        # block too large
+    assert L.memosight_attn_workspace_bytes(1, 4, 2, 64, 10, 32769) == 0        # block too large
     assert L.memosight_attn_workspace_bytes(1, 4, 2, 64, 10, 4) > 256
 
     def params(**kw):
@@ -67,7 +67,7 @@ def test_host_side_validation_codes():
         return p
     assert L.memosight_attn_step(C.byref(params(n_q_heads=5)), None) == ms.MS_ERR_INVALID_ARG
     assert L.memosight_attn_step(C.byref(params(head_dim=48)), None) == ms.MS_ERR_UNSUPPORTED_SHAPE
-    assert L.memosight_attn_step(C.byref(params(max_nq=257)), None) == ms.MS_ERR_UNSUPPORTED_SHAPE
+    assert L.memosight_attn_step(C.byref(params(max_nq=32769)), None) == ms.MS_ERR_UNSUPPORTED_SHAPE
     assert L.memosight_attn_step(C.byref(params()), None) == ms.MS_ERR_INVALID_ARG       # null pointers
     fake = 0x1000
     full = dict(k_cache=fake, v_cache=fake, kv_off=fake, kv_len=fake, q_off=fake, n_cand=fake, q=fake,

@@ -80,7 +80,14 @@ def test_large_block_equals_the_same_tokens_as_small_blocks():
 
 def test_block_size_limits():
     P = random_problem(1, 8, 2, 128, [10], [16], [16], seed=1)
-    assert ms.memosight_attn_workspace_bytes(1, 8, 2, 128, 10, 257) == 0
+    assert ms.memosight_attn_workspace_bytes(1, 8, 2, 128, 10, 32769) == 0
     assert ms.memosight_attn_workspace_bytes(1, 8, 2, 128, 10, 256) > ms.memosight_attn_workspace_bytes(1, 8, 2, 128, 10, 16)
     # head_dim 64 has no large-block tensor-core kernel: the general kernel serves it
     check_attn(random_problem(1, 4, 2, 64, [200], [40], [40], seed=2), "D=64 large block")
+
+
+def test_prefill_sized_blocks():
+    # Algorithm 1, Prefill: the prompt is one causal block; with an empty cache, and as a chunk
+    # behind an already cached part, for two sequences of different length
+    check_attn(random_problem(2, 8, 2, 128, [0, 0], [1500, 700], [1500, 700], seed=51), "prefill, empty cache")
+    check_attn(random_problem(2, 8, 2, 128, [1000, 3], [1024, 257], [1024, 257], seed=52), "chunked prefill")
