@@ -15,7 +15,7 @@
 // share every tile: warpgroup g takes key columns [64g, 64g+64) of the scores and, for rescales
 // and the epilogue, output columns [64g, 64g+64) of its rows.  A row's reference maximum is the
 // exact maximum of the unit's first tile (both halves, exchanged through shared memory) and only
-// moves when a score exceeds it by 2^48; the eight softmax warps agree on that through one
+// moves when a score exceeds it by about 2^48 (seen in the tile's row sum); the eight softmax warps agree on that through one
 // bounded mbarrier round per tile.  Row sums are kept per thread and added up at the unit's end.
 // Schedule: the flat list of all tiles of all units, cut into one contiguous range per
 // persistent CTA; a unit cut across CTAs leaves (m, l, O) partials that attn_big_merge_kernel
@@ -29,7 +29,7 @@ constexpr int kBThreads = 384;    // warp 0: TMA, warp 1: MMA issue, 4-7 and 8-1
 constexpr int kBD = 128;
 constexpr uint32_t kBCols = 512;  // S0 | S1 | O
 constexpr uint32_t kBColS = 0, kBColO = 256;
-constexpr float kBGrowLimit = 48.f;
+constexpr float kBGrowSum = 281474976710656.f;   // 2^48: a partial row sum this large moves the reference
 constexpr int kBKv = 4;                           // K/V buffers in the ring
 constexpr int kBKvBytes = kTile * kBD * 2;        // 32 KB
 constexpr uint32_t kBHalf = kTile * 128;          // bytes between 64-column halves of a tile
@@ -166,21 +166,20 @@ __device__ __host__ inline size_t big_slot_floats() { return static_cast<size_t>
 template <bool kMasked>
 __device__ __forceinline__ void big_load_scores(uint32_t s_addr, float (&v)[64], int col0, int nv, bool is_step,
                                                 int tok, int key0, int n_c, int anc) {
+  uint32_t raw0[32], raw1[32];
+  tmem_ld32(s_addr, raw0);
+  tmem_ld32(s_addr + 32, raw1);
+  tmem_ld_wait(raw0);
+  tmem_ld_wait(raw1);
 #pragma unroll
-  for (int c = 0; c < 2; ++c) {
-    uint32_t raw[32];
-    tmem_ld32(s_addr + c * 32, raw);
-    tmem_ld_wait(raw);
-#pragma unroll
-    for (int e = 0; e < 32; ++e) {
-      float s = __uint_as_float(raw[e]);
-      if (kMasked) {
-        bool vis = col0 + c * 32 + e < nv;
-        if (is_step) vis = vis && step_key_visible(tok, key0 + c * 32 + e, n_c, anc);
-        s = vis ? s : -INFINITY;
-      }
-      v[c * 32 + e] = s;
+  for (int e = 0; e < 64; ++e) {
+    float s = __uint_as_float(e < 32 ? raw0[e & 31] : raw1[e & 31]);
+    if (kMasked) {
+      bool vis = col0 + e < nv;
+      if (is_step) vis = vis && step_key_visible(tok, key0 + e, n_c, anc);
+      s = vis ? s : -INFINITY;
     }
+    v[e] = s;
   }
 }
 __device__ __forceinline__ float max64(const float (&v)[64]) {
@@ -462,15 +461,34 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
         m_ref = (m == -INFINITY) ? 0.f : m * a.scale_log2;
         l_part = 0.f;
       }
+      // p = 2^(s*scale - m_ref) as bf16 into this row of the P tile (half g = this group's 64 keys);
+      // returns the row's partial sum over those keys
+      const uint32_t p_row = sb + kBOffP + pb * kBPBytes + wg * kBHalf + r * 128;
+      auto p_pass = [&]() -> float {
+        float ls[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int j = 0; j < 64; ++j) v[j] = fmaf(v[j], a.scale_log2, -m_ref);
-      const float tmaxx = max64(v);
-      if (w.piece_j > 0 && __any_sync(0xffffffffu, row_ok && tmaxx > kBGrowLimit) && lane == 0)
+        for (int c = 0; c < 8; ++c) {
+          float p[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            p[e] = ex2(fmaf(v[c * 8 + e], a.scale_log2, -m_ref));
+            ls[e & 3] += p[e];
+          }
+          const uint32_t addr = p_row + ((c ^ rx) << 4);
+          asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(pack2(p[0], p[1])),
+                       "r"(pack2(p[2], p[3])), "r"(pack2(p[4], p[5])), "r"(pack2(p[6], p[7]))
+                       : "memory");
+        }
+        return (ls[0] + ls[1]) + (ls[2] + ls[3]);
+      };
+      float tsum = p_pass();
+      // A score that outgrew the row reference by ~2^48 shows in the sum (so do inf and NaN); the
+      // eight warps agree on it before anyone hands P over
+      if (w.piece_j > 0 && __any_sync(0xffffffffu, row_ok && !(tsum < kBGrowSum)) && lane == 0)
         *grow_flag = it + 1;
       if (!sync8()) { ok = false; break; }
       if (*grow_flag == it + 1) {
         // ---- rare: move the row references up; rescale O (this group's 64 columns) and the sums ----
-        load_scores();
         s_mx[wg * 128 + r] = max64(v);
         if (!sync8()) { ok = false; break; }
         const float m = fmaxf(s_mx[r], s_mx[128 + r]);
@@ -490,29 +508,10 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
           tmem_st32(lane_addr + kBColO + wg * 64 + c * 32, o);
         }
         asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-#pragma unroll
-        for (int j = 0; j < 64; ++j) v[j] = fmaf(v[j], a.scale_log2, -m_ref);
+        tsum = p_pass();
         if (!sync8()) { ok = false; break; }     // s_mx may be rewritten from here on
       }
-      // p = 2^x as bf16 into this row of the P tile (half g = this group's 64 keys)
-      {
-        const uint32_t p_row = sb + kBOffP + pb * kBPBytes + wg * kBHalf + r * 128;
-        float ls[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          float p[8];
-#pragma unroll
-          for (int e = 0; e < 8; ++e) {
-            p[e] = ex2(v[c * 8 + e]);
-            ls[e & 3] += p[e];
-          }
-          const uint32_t addr = p_row + ((c ^ rx) << 4);
-          asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(pack2(p[0], p[1])),
-                       "r"(pack2(p[2], p[3])), "r"(pack2(p[4], p[5])), "r"(pack2(p[6], p[7]))
-                       : "memory");
-        }
-        l_part += (ls[0] + ls[1]) + (ls[2] + ls[3]);
-      }
+      l_part += tsum;
       fence_async_smem();
       tc_fence_before();
       __syncwarp();
