@@ -160,8 +160,7 @@ typedef struct memosight_attn_params {
   void* ev_split_end;        /* ... and right after the split-KV kernel (NULL: not recorded)   */
 } memosight_attn_params;
 
-/* Scratch size for memosight_attn_step with these bounds (0 on invalid input).
- * It does not depend on the cache length: the split-KV partials are per CTA. */
+/* Scratch size for memosight_attn_step with these bounds (0 on invalid input). */
 MS_API size_t memosight_attn_workspace_bytes(int32_t batch, int32_t n_q_heads, int32_t n_kv_heads,
                                       int32_t head_dim, int32_t max_kv_len, int32_t max_nq);
 
@@ -173,8 +172,9 @@ MS_API size_t memosight_attn_workspace_bytes(int32_t batch, int32_t n_q_heads, i
  * (Sec. 2.1.2, Algorithm 1), and the prefill of a prompt is one causal block against an empty
  * or partly filled cache (Algorithm 1, Prefill) -- take the large-block tcgen05 kernel when D
  * is 128.  Anything
- * else inside the limits takes the slower general kernel.  Pass the max_nq the workspace was
- * sized for: the workspace of a large-block call is bigger.
+ * else inside the limits takes the slower general kernel.  Size the workspace with the very
+ * batch, head counts, max_kv_len and max_nq of the call: a large-block call needs a different
+ * amount than a step-block call.
  * The workspace may be reused by the next call on the same stream; two calls
  * that overlap on the GPU need two workspaces. */
 MS_API int32_t memosight_attn_step(const memosight_attn_params* params, memosight_stream_t stream);

@@ -55,7 +55,8 @@ extern "C" size_t memosight_attn_workspace_bytes(int32_t batch, int32_t n_q_head
   const int G = n_q_heads / n_kv_heads;
   int n_ctas = ms::attn_mma_grid();
   if (n_ctas <= 0) n_ctas = 256;   // no device visible: answer for the largest part we target
-  if (ms::attn_umma_big_supports(head_dim, G, max_nq)) return ms::attn_umma_big_workspace_bytes(n_ctas);
+  if (ms::attn_umma_big_supports(head_dim, G, max_nq))
+    return ms::attn_umma_big_workspace_bytes(batch, n_kv_heads, G, max_nq, max_kv_len, n_ctas);
   if (!fast_path_shape(head_dim, G, max_nq)) return ms::kWsHeaderBytes;
   const int rows_pad = (max_nq * G + 15) & ~15;
   return ms::attn_mma_workspace_bytes(head_dim, rows_pad, n_ctas);

@@ -54,7 +54,7 @@ int32_t launch_attn_umma_t(const AttnArgs& a, cudaStream_t st);
 // tcgen05 path for large blocks (17..256 tokens per block, head_dim 128): the block is cut
 // into row tiles; own schedule, workspace size and merge kernel.
 bool attn_umma_big_supports(int D, int G, int max_nq);
-size_t attn_umma_big_workspace_bytes(int n_ctas);
+size_t attn_umma_big_workspace_bytes(int B, int H_kv, int G, int max_nq, int max_kv_len, int n_ctas);
 int32_t launch_attn_umma_big(const AttnArgs& a, cudaStream_t st);
 
 }  // namespace ms

@@ -17,9 +17,9 @@
 // exact maximum of the unit's first tile (both halves, exchanged through shared memory) and only
 // moves when a score exceeds it by about 2^48 (seen in the tile's row sum); the eight softmax warps agree on that through one
 // bounded mbarrier round per tile.  Row sums are kept per thread and added up at the unit's end.
-// Schedule: the flat list of all tiles of all units, cut into one contiguous range per
-// persistent CTA; a unit cut across CTAs leaves (m, l, O) partials that attn_big_merge_kernel
-// combines.  Every wait is bounded (status word in the workspace, as in the other paths).
+// Schedule: work items dealt round-robin to the persistent CTAs so that the row tiles of one K/V
+// chunk run side by side (see below); every wait is bounded (status word in the workspace, as in
+// the other paths).
 #include "attn_umma_common.cuh"
 
 namespace ms {
@@ -48,9 +48,17 @@ enum : int {
 static_assert(kBbCount * 8 <= kBMiscScalars, "barriers overflow their slot");
 
 // ---------------------------------------------------------------- schedule
+//
+// Work items are (sequence, KV head, chunk of the unit's tiles, row tile), enumerated in that
+// order with the row tile fastest, and dealt to the persistent CTAs round-robin: at any moment
+// neighbouring CTAs work on the row tiles of the same K/V chunk, so a K/V tile that several row
+// tiles need is fetched from HBM once and found in L2 by the others.  A unit's tiles (cache tiles,
+// then the step-local key tiles up to the row tile's last token) are cut into `nsplit` chunks only
+// when there are too few units to fill the machine; a chunked unit leaves one (m, l, O) partial per
+// chunk for attn_big_merge_kernel.
 
 struct BigSeq {
-  int L, n_q, r0, n_c, cache_tiles, n_rt, tph;   // tph: tiles of one KV head (all row tiles)
+  int L, n_q, r0, n_c, cache_tiles, n_rt;
   long long slot_off;
 };
 __device__ __forceinline__ int big_step_tiles(const BigSeq& s, int rt, int tpt) {
@@ -64,12 +72,12 @@ __device__ __forceinline__ void big_seq(const AttnArgs& a, int b, int tpt, BigSe
   s.slot_off = a.kv_off[b];
   s.cache_tiles = (s.L + kTile - 1) / kTile;
   s.n_rt = (s.n_q + tpt - 1) / tpt;
-  int t = s.n_rt * s.cache_tiles;
-  for (int rt = 0; rt < s.n_rt; ++rt) t += big_step_tiles(s, rt, tpt);
-  s.tph = t;
 }
-// Exclusive prefix sum of tph over the batch into pre[0..B] (shared memory).
-__device__ void big_build_prefix(const AttnArgs& a, int tpt, int* pre, int* scratch) {
+
+// pre[0..B]: exclusive prefix sum of the sequences' row-tile counts (one CTA).
+__global__ void __launch_bounds__(256)
+attn_big_plan_kernel(const AttnArgs a, int tpt, int* __restrict__ pre) {
+  __shared__ int scratch[256];
   const int nt = blockDim.x, tid = threadIdx.x;
   const int per = (a.B + nt - 1) / nt;
   const int lo = min(a.B, tid * per), hi = min(a.B, lo + per);
@@ -77,7 +85,7 @@ __device__ void big_build_prefix(const AttnArgs& a, int tpt, int* pre, int* scra
   for (int b = lo; b < hi; ++b) {
     BigSeq s;
     big_seq(a, b, tpt, s);
-    sum += s.tph;
+    sum += s.n_rt;
   }
   scratch[tid] = sum;
   __syncthreads();
@@ -87,75 +95,73 @@ __device__ void big_build_prefix(const AttnArgs& a, int tpt, int* pre, int* scra
     BigSeq s;
     big_seq(a, b, tpt, s);
     pre[b] = base;
-    base += s.tph;
+    base += s.n_rt;
   }
   if (tid == nt - 1) pre[a.B] = base;
-  __syncthreads();
 }
 
 struct BigWalk {
   BigSeq s;
-  int b, h, rt, ti, tiles_u, tpt;
-  int it, n_iter, piece_idx, piece_j, slot;
-  bool open, first, last;
+  int b, h, rt, ti, ti_lo, ti_hi, tpt;
+  int item, n_items, nsplit;
+  int it, piece_idx, piece_j, slot;
+  bool first, last, done;
   int step_idx, nvalid;     // step_idx < 0: cache tile
 };
-__device__ __forceinline__ void bwalk_init(const AttnArgs& a, BigWalk& w, int tpt, int b0, long long rel,
-                                           int n_iter) {
-  w.tpt = tpt;
-  w.b = b0;
-  big_seq(a, b0, tpt, w.s);
-  w.h = static_cast<int>(rel / w.s.tph);
-  int rem = static_cast<int>(rel - static_cast<long long>(w.h) * w.s.tph);
-  w.rt = 0;
+// Moves to this CTA's next non-empty item (items are visited with stride gridDim.x).
+__device__ __forceinline__ void bwalk_advance(const AttnArgs& a, BigWalk& w, const int* __restrict__ pre) {
   for (;;) {
-    const int tu = w.s.cache_tiles + big_step_tiles(w.s, w.rt, tpt);
-    if (rem < tu || w.rt + 1 >= w.s.n_rt) { w.tiles_u = tu; break; }
-    rem -= tu;
-    ++w.rt;
+    w.item += static_cast<int>(gridDim.x);
+    if (w.item >= w.n_items) { w.done = true; return; }
+    const int per_rt = a.H_kv * w.nsplit;                 // items per row tile of a sequence
+    int lo = 0, hi = a.B;
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (static_cast<long long>(pre[mid]) * per_rt <= w.item) lo = mid; else hi = mid;
+    }
+    w.b = lo;
+    big_seq(a, lo, w.tpt, w.s);
+    if (w.s.n_rt == 0) continue;                          // cannot happen for a valid index; stay safe
+    int j = w.item - pre[lo] * per_rt;
+    const int per_head = w.nsplit * w.s.n_rt;
+    w.h = j / per_head;
+    j -= w.h * per_head;
+    const int chunk = j / w.s.n_rt;
+    w.rt = j - chunk * w.s.n_rt;
+    const int tiles_u = w.s.cache_tiles + big_step_tiles(w.s, w.rt, w.tpt);
+    w.ti_lo = static_cast<int>(static_cast<long long>(tiles_u) * chunk / w.nsplit);
+    w.ti_hi = static_cast<int>(static_cast<long long>(tiles_u) * (chunk + 1) / w.nsplit);
+    if (w.ti_lo < w.ti_hi) break;
   }
-  w.ti = rem;
+  w.ti = w.ti_lo;
+}
+__device__ __forceinline__ void bwalk_init(const AttnArgs& a, BigWalk& w, int tpt, int nsplit, const int* pre) {
+  w.tpt = tpt;
+  w.nsplit = nsplit;
+  w.n_items = pre[a.B] * a.H_kv * nsplit;
+  w.item = static_cast<int>(blockIdx.x) - static_cast<int>(gridDim.x);
   w.it = 0;
-  w.n_iter = n_iter;
   w.piece_idx = -1;
   w.piece_j = 0;
   w.slot = 0;
-  w.open = false;
+  w.done = false;
+  bwalk_advance(a, w, pre);
 }
 __device__ __forceinline__ void bwalk_tile(BigWalk& w) {
-  const int left = w.n_iter - w.it;
-  w.first = !w.open;
+  w.first = (w.ti == w.ti_lo);
   if (w.first) {
-    const bool whole = (w.ti == 0) && (left >= w.tiles_u);
-    w.slot = whole ? -1 : 2 * static_cast<int>(blockIdx.x) + (w.it == 0 ? 0 : 1);
-    w.open = true;
+    w.slot = (w.nsplit == 1) ? -1 : w.item;
     w.piece_idx += 1;
     w.piece_j = 0;
   }
   w.step_idx = w.ti - w.s.cache_tiles;
-  w.last = (w.ti == w.tiles_u - 1) || left == 1;
+  w.last = (w.ti == w.ti_hi - 1);
   w.nvalid = w.step_idx >= 0 ? min(kTile, w.s.n_q - w.step_idx * kTile) : min(kTile, w.s.L - w.ti * kTile);
 }
-__device__ __forceinline__ void bwalk_next(const AttnArgs& a, BigWalk& w) {
-  if (w.last) w.open = false;
+__device__ __forceinline__ void bwalk_next(const AttnArgs& a, BigWalk& w, const int* __restrict__ pre) {
   w.piece_j += 1;
   w.it += 1;
-  if (++w.ti == w.tiles_u) {
-    w.ti = 0;
-    if (++w.rt == w.s.n_rt) {
-      w.rt = 0;
-      if (++w.h == a.H_kv) {
-        w.h = 0;
-        if (w.it < w.n_iter) {
-          do {
-            ++w.b;
-            big_seq(a, w.b, w.tpt, w.s);
-          } while (w.s.tph == 0 && w.b + 1 < a.B);
-        }
-      }
-    }
-    w.tiles_u = w.s.cache_tiles + big_step_tiles(w.s, w.rt, w.tpt);
-  }
+  if (++w.ti == w.ti_hi) bwalk_advance(a, w, pre);
 }
 
 __device__ __host__ inline size_t big_slot_floats() { return static_cast<size_t>(kTile) * (kBD + 2); }
@@ -197,7 +203,7 @@ __global__ void __launch_bounds__(kBThreads, 1)
 attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
                      const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_ks,
                      const __grid_constant__ CUtensorMap map_vs, const __grid_constant__ CUtensorMap map_q,
-                     int tpt) {
+                     int tpt, int nsplit) {
   constexpr int D = kBD, HALVES = 2, KSTEPS = D / 16;
   extern __shared__ __align__(1024) uint8_t smem[];
   const uint32_t sb = smem_u32(smem);
@@ -218,26 +224,17 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
   }
   const int rows_box = tpt * a.G;
 
-  // ---- schedule (the prefix lives where the buffers will be) ----
-  int* s_pre = reinterpret_cast<int*>(smem);
-  int* s_scratch = s_pre + a.B + 1;
-  big_build_prefix(a, tpt, s_pre, s_scratch);
-  const long long n_tiles = static_cast<long long>(s_pre[a.B]) * a.H_kv;
-  const long long t0 = n_tiles * blockIdx.x / gridDim.x;
-  const long long t1 = n_tiles * (blockIdx.x + 1) / gridDim.x;
-  const int n_iter = static_cast<int>(t1 - t0);
-  if (blockIdx.x == 0) {
-    for (int i = threadIdx.x; i <= a.B; i += blockDim.x) ws_pre[i] = s_pre[i];
-  }
+  // ---- schedule: this CTA's items, and how many tiles they hold ----
+  const int* __restrict__ pre = ws_pre;
   BigWalk w0;
-  w0.n_iter = 0;
-  if (n_iter > 0) {
-    int lo = 0, hi = a.B;
-    while (hi - lo > 1) {
-      const int mid = (lo + hi) >> 1;
-      if (static_cast<long long>(s_pre[mid]) * a.H_kv <= t0) lo = mid; else hi = mid;
+  bwalk_init(a, w0, tpt, nsplit, pre);
+  int n_iter = 0;
+  {
+    BigWalk wc = w0;
+    while (!wc.done) {
+      n_iter += wc.ti_hi - wc.ti_lo;
+      bwalk_advance(a, wc, pre);
     }
-    bwalk_init(a, w0, tpt, lo, t0 - static_cast<long long>(s_pre[lo]) * a.H_kv, n_iter);
   }
   if (threadIdx.x == 0) {
     for (int i = 0; i < kBKv; ++i) {
@@ -257,7 +254,7 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
     *grow_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  __syncthreads();   // the prefix has been consumed
+  __syncthreads();
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
                      smem_u32(tmem_slot)), "r"(kBCols)
@@ -312,7 +309,7 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
         ++uses;
       }
       if (!ok) break;
-      bwalk_next(a, w);
+      bwalk_next(a, w, pre);
     }
     for (int u = uses > kBKv ? uses - kBKv : 0; u < uses; ++u)
       (void)mbar_wait(bars + 8 * (kBbKvFull + u % kBKv), (u / kBKv) & 1, abort_flag, status);
@@ -345,7 +342,7 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
       umma_commit(bars + 8 * (kBbSFull + (it & 1)));
       if (wq.last) umma_commit(bars + 8 * kBbQEmpty);
       rk.step(2);
-      bwalk_next(a, wq);
+      bwalk_next(a, wq, pre);
       return true;
     };
     ok = issue_qk();
@@ -377,7 +374,7 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
       umma_commit(bars + 8 * (kBbKvEmpty + rv.buf));
       umma_commit(bars + 8 * (kBbPvDone + (it & 1)));
       rv.step(2);
-      bwalk_next(a, wp);
+      bwalk_next(a, wp, pre);
     }
     if (!ok) {
       umma_commit(bars + 8 * kBbDrain);
@@ -561,7 +558,7 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
         }
         tc_fence_before();   // the reads of O are ordered before the next unit's first PV product
       }
-      bwalk_next(a, w);
+      bwalk_next(a, w, pre);
     }
   }
 
@@ -575,51 +572,43 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
   }
 }
 
-// One CTA per (sequence, KV head, row tile) unit that the split kernel cut across CTAs; one warp
-// per packed row folds the pieces' (m, l) with shuffles and accumulates its output columns.
+// One CTA per (sequence, KV head, row tile) unit of a chunked launch; one warp per packed row
+// folds the chunks' (m, l) with shuffles and accumulates its output columns.
 __global__ void __launch_bounds__(128)
-attn_big_merge_kernel(const AttnArgs a, int tpt, int max_rt, int n_ctas) {
+attn_big_merge_kernel(const AttnArgs a, int tpt, int max_rt, int nsplit) {
   constexpr int D = kBD, E = D / 32;
   int u = blockIdx.x;
   const int rt = u % max_rt; u /= max_rt;
   const int h = u % a.H_kv;
   const int b = u / a.H_kv;
-  const int* ws_pre = reinterpret_cast<const int*>(reinterpret_cast<const uint8_t*>(a.workspace) +
-                                                   kWsHeaderBytes);
+  const int* pre = reinterpret_cast<const int*>(reinterpret_cast<const uint8_t*>(a.workspace) + kWsHeaderBytes);
   const float* ws_slots = reinterpret_cast<const float*>(
       reinterpret_cast<const uint8_t*>(a.workspace) + kWsHeaderBytes + ws_prefix_bytes());
   BigSeq s;
   big_seq(a, b, tpt, s);
-  if (rt >= s.n_rt || s.tph == 0) return;
-  const long long n_tiles = static_cast<long long>(ws_pre[a.B]) * a.H_kv;
-  long long u0 = static_cast<long long>(ws_pre[b]) * a.H_kv + static_cast<long long>(h) * s.tph;
-  for (int x = 0; x < rt; ++x) u0 += s.cache_tiles + big_step_tiles(s, x, tpt);
-  const long long u1 = u0 + s.cache_tiles + big_step_tiles(s, rt, tpt);
-  const int c_lo = static_cast<int>(((u0 + 1) * n_ctas - 1) / n_tiles);
-  const int c_hi = static_cast<int>((u1 * n_ctas - 1) / n_tiles);
-  if (c_lo == c_hi) return;                      // whole unit inside one CTA: already written
+  if (rt >= s.n_rt) return;
+  const int tiles_u = s.cache_tiles + big_step_tiles(s, rt, tpt);
+  // slot of chunk k = its item index; a chunk without tiles has no partial
+  const long long item0 = static_cast<long long>(pre[b]) * a.H_kv * nsplit +
+                          static_cast<long long>(h) * nsplit * s.n_rt + rt;
   const int tok0 = rt * tpt;
   const int rows = (min(s.n_q, tok0 + tpt) - tok0) * a.G;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const size_t slot_floats = big_slot_floats();
   for (int r = warp; r < rows; r += 4) {
     float M = -INFINITY;
-    for (int c = c_lo + lane; c <= c_hi; c += 32) {
-      const long long s0 = n_tiles * c / n_ctas, s1 = n_tiles * (c + 1) / n_ctas;
-      if (s1 <= s0) continue;
-      const int slot = 2 * c + ((s0 >= u0) ? 0 : 1);
-      M = fmaxf(M, ws_slots[slot * slot_floats + static_cast<size_t>(kTile) * D + r]);
+    if (lane < nsplit) {
+      const bool has = static_cast<long long>(tiles_u) * lane / nsplit < static_cast<long long>(tiles_u) * (lane + 1) / nsplit;
+      if (has) M = ws_slots[(item0 + static_cast<long long>(lane) * s.n_rt) * slot_floats + static_cast<size_t>(kTile) * D + r];
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
     float Lsum = 0.f, acc[E];
 #pragma unroll
     for (int e = 0; e < E; ++e) acc[e] = 0.f;
-    for (int c = c_lo; c <= c_hi; ++c) {
-      const long long s0 = n_tiles * c / n_ctas, s1 = n_tiles * (c + 1) / n_ctas;
-      if (s1 <= s0) continue;
-      const int slot = 2 * c + ((s0 >= u0) ? 0 : 1);
-      const float* sp = ws_slots + slot * slot_floats;
+    for (int k = 0; k < nsplit; ++k) {
+      if (static_cast<long long>(tiles_u) * k / nsplit >= static_cast<long long>(tiles_u) * (k + 1) / nsplit) continue;
+      const float* sp = ws_slots + (item0 + static_cast<long long>(k) * s.n_rt) * slot_floats;
       const float m = sp[static_cast<size_t>(kTile) * D + r];
       const float l = sp[static_cast<size_t>(kTile) * D + kTile + r];
       const float wgt = (m == -INFINITY) ? 0.f : exp2f(m - M);
@@ -638,24 +627,48 @@ attn_big_merge_kernel(const AttnArgs a, int tpt, int max_rt, int n_ctas) {
   }
 }
 
+// Chunks per unit, from a small cost model in units of one tile's time: items are dealt
+// round-robin and take about the same time, so a launch lasts ceil(items / CTAs) rounds of
+// (tiles per item + a fixed start-up/epilogue cost); chunked launches also pay for writing and
+// merging one partial per item.  Chunking is chosen only when it wins clearly.
+int big_nsplit(int B, int H_kv, int max_rt, int n_ctas, int max_kv_len) {
+  const long long units = static_cast<long long>(B) * H_kv * max_rt;
+  if (units == 0) return 1;
+  const double tiles = max_kv_len / kTile + 2.0;
+  int best = 1;
+  double best_cost = 0.0;
+  for (int ns = 1; ns <= 16; ++ns) {
+    if (ns > 1 && tiles / ns < 8.0) break;
+    const long long items = units * ns;
+    const long long rounds = (items + n_ctas - 1) / n_ctas;
+    const double cost = rounds * (tiles / ns + 4.0) + (ns > 1 ? 0.015 * items : 0.0);
+    if (ns == 1 || cost < 0.92 * best_cost) { best = ns; best_cost = cost; }
+  }
+  return best;
+}
+
 }  // namespace
 
 bool attn_umma_big_supports(int D, int G, int max_nq) {
   return D == kBD && G >= 1 && G <= kMaxGroup && max_nq > kMaxNq && max_nq <= kMaxNqBig;
 }
 
-size_t attn_umma_big_workspace_bytes(int n_ctas) {
-  return kWsHeaderBytes + ws_prefix_bytes() + static_cast<size_t>(2) * n_ctas * big_slot_floats() * sizeof(float);
+size_t attn_umma_big_workspace_bytes(int B, int H_kv, int G, int max_nq, int max_kv_len, int n_ctas) {
+  const int tpt = kTile / G, max_rt = (max_nq + tpt - 1) / tpt;
+  const int nsplit = big_nsplit(B, H_kv, max_rt, n_ctas, max_kv_len);
+  const size_t slots = nsplit > 1 ? static_cast<size_t>(B) * H_kv * max_rt * nsplit : 0;
+  return kWsHeaderBytes + ws_prefix_bytes() + slots * big_slot_floats() * sizeof(float);
 }
 
 int32_t launch_attn_umma_big(const AttnArgs& a, cudaStream_t st) {
   if (a.B == 0 || a.T == 0) return MS_OK;
   if (!attn_umma_big_supports(a.D, a.G, a.max_nq)) return MS_ERR_UNSUPPORTED_SHAPE;
-  if (static_cast<int>((a.B + 1 + kBThreads) * sizeof(int)) > kBOffMisc) return MS_ERR_UNSUPPORTED_SHAPE;
   const int tpt = kTile / a.G;                   // tokens per row tile
   const int max_rt = (a.max_nq + tpt - 1) / tpt;
   const int grid = attn_mma_grid();
   if (grid <= 0) return cuda_status(cudaErrorNoDevice);
+  const int nsplit = big_nsplit(a.B, a.H_kv, max_rt, grid, a.max_kv_len);
+  if (static_cast<long long>(a.B) * a.H_kv * max_rt * nsplit > 0x7fffffffLL) return MS_ERR_UNSUPPORTED_SHAPE;
   CUtensorMap mk, mv, mks, mvs, mq;
   const bool ok =
       make_map(&mk, a.k_cache, a.D, static_cast<uint64_t>(a.n_slots), a.H_kv, a.D, a.kv_head_stride, kTile, 1) &&
@@ -671,13 +684,18 @@ int32_t launch_attn_umma_big(const AttnArgs& a, cudaStream_t st) {
     MS_CUDA_TRY(cudaFuncSetAttribute(attn_umma_big_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kBSmem));
     configured[dev] = true;
   }
+  int* pre = reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(a.workspace) + kWsHeaderBytes);
+  attn_big_plan_kernel<<<1, 256, 0, st>>>(a, tpt, pre);
+  MS_LAUNCH_CHECK();
   if (a.ev_split_begin) MS_CUDA_TRY(cudaEventRecord(a.ev_split_begin, st));
-  attn_umma_big_kernel<<<grid, kBThreads, kBSmem, st>>>(a, mk, mv, mks, mvs, mq, tpt);
+  attn_umma_big_kernel<<<grid, kBThreads, kBSmem, st>>>(a, mk, mv, mks, mvs, mq, tpt, nsplit);
   MS_LAUNCH_CHECK();
   if (a.ev_split_end) MS_CUDA_TRY(cudaEventRecord(a.ev_split_end, st));
-  const long long units = static_cast<long long>(a.B) * a.H_kv * max_rt;
-  attn_big_merge_kernel<<<static_cast<unsigned>(units), 128, 0, st>>>(a, tpt, max_rt, grid);
-  MS_LAUNCH_CHECK();
+  if (nsplit > 1) {
+    const long long units = static_cast<long long>(a.B) * a.H_kv * max_rt;
+    attn_big_merge_kernel<<<static_cast<unsigned>(units), 128, 0, st>>>(a, tpt, max_rt, nsplit);
+    MS_LAUNCH_CHECK();
+  }
   return MS_OK;
 }
 
