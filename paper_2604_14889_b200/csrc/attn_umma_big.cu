@@ -25,8 +25,11 @@
 namespace ms {
 namespace {
 
-constexpr int kBThreads = 384;    // warp 0: TMA, warp 1: MMA issue, 4-7 and 8-11: softmax warpgroups
+constexpr int kBWg = 2;                           // softmax warpgroups: each takes 128 / kBWg key columns of a tile
+constexpr int kBCw = kTile / kBWg;
+constexpr int kBThreads = 128 + 128 * kBWg;       // warp 0: TMA, warp 1: MMA issue, warps 4..: softmax warpgroups
 constexpr int kBD = 128;
+static_assert(kBCw % 32 == 0 && kBD / kBWg == kBCw, "a warpgroup's score and output columns are whole 32-column loads");
 constexpr uint32_t kBCols = 512;  // S0 | S1 | O
 constexpr uint32_t kBColS = 0, kBColO = 256;
 constexpr float kBGrowSum = 281474976710656.f;   // 2^48: a partial row sum this large moves the reference
@@ -36,8 +39,8 @@ constexpr uint32_t kBHalf = kTile * 128;          // bytes between 64-column hal
 constexpr int kBQBytes = 2 * kBHalf, kBPBytes = 2 * kBHalf;
 constexpr int kBOffQ = 0, kBOffP = kBQBytes, kBOffKv = kBOffP + 2 * kBPBytes;
 constexpr int kBOffMisc = kBOffKv + kBKv * kBKvBytes;
-// misc: barriers | scalars | mx[2][128] | lpart[2][128]
-constexpr int kBMiscScalars = 256, kBMiscMx = 512, kBMiscL = 1536, kBMiscBytes = 2560;
+// misc: barriers | scalars | mx[kBWg][128] and lpart[kBWg][128] (one region: they are never live together)
+constexpr int kBMiscScalars = 256, kBMiscMx = 512, kBMiscL = 512, kBMiscBytes = 512 + kBWg * kTile * 4;
 constexpr int kBSmem = kBOffMisc + kBMiscBytes;
 static_assert(kBSmem <= 227 * 1024, "shared memory budget");
 
@@ -170,16 +173,16 @@ __device__ __host__ inline size_t big_slot_floats() { return static_cast<size_t>
 // invisible keys (past the valid length; on a step-local tile by the (n_cand, anchor) rule)
 // become -inf.
 template <bool kMasked>
-__device__ __forceinline__ void big_load_scores(uint32_t s_addr, float (&v)[64], int col0, int nv, bool is_step,
+__device__ __forceinline__ void big_load_scores(uint32_t s_addr, float (&v)[kBCw], int col0, int nv, bool is_step,
                                                 int tok, int key0, int n_c, int anc) {
-  uint32_t raw0[32], raw1[32];
-  tmem_ld32(s_addr, raw0);
-  tmem_ld32(s_addr + 32, raw1);
-  tmem_ld_wait(raw0);
-  tmem_ld_wait(raw1);
+  uint32_t raw[kBCw / 32][32];
 #pragma unroll
-  for (int e = 0; e < 64; ++e) {
-    float s = __uint_as_float(e < 32 ? raw0[e & 31] : raw1[e & 31]);
+  for (int c = 0; c < kBCw / 32; ++c) tmem_ld32(s_addr + c * 32, raw[c]);
+#pragma unroll
+  for (int c = 0; c < kBCw / 32; ++c) tmem_ld_wait(raw[c]);
+#pragma unroll
+  for (int e = 0; e < kBCw; ++e) {
+    float s = __uint_as_float(raw[e >> 5][e & 31]);
     if (kMasked) {
       bool vis = col0 + e < nv;
       if (is_step) vis = vis && step_key_visible(tok, key0 + e, n_c, anc);
@@ -188,12 +191,12 @@ __device__ __forceinline__ void big_load_scores(uint32_t s_addr, float (&v)[64],
     v[e] = s;
   }
 }
-__device__ __forceinline__ float max64(const float (&v)[64]) {
+__device__ __forceinline__ float max_cols(const float (&v)[kBCw]) {
   float m[8];
 #pragma unroll
   for (int j = 0; j < 8; ++j) m[j] = v[j];
 #pragma unroll
-  for (int j = 8; j < 64; ++j) m[j & 7] = fmaxf(m[j & 7], v[j]);
+  for (int j = 8; j < kBCw; ++j) m[j & 7] = fmaxf(m[j & 7], v[j]);
   return fmaxf(fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3])), fmaxf(fmaxf(m[4], m[5]), fmaxf(m[6], m[7])));
 }
 
@@ -211,8 +214,8 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kBOffMisc + kBMiscScalars);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kBOffMisc + kBMiscScalars + 8);
   volatile int* grow_flag = reinterpret_cast<volatile int*>(smem + kBOffMisc + kBMiscScalars + 16);
-  float* s_mx = reinterpret_cast<float*>(smem + kBOffMisc + kBMiscMx);      // [2][128]
-  float* s_lp = reinterpret_cast<float*>(smem + kBOffMisc + kBMiscL);       // [2][128]
+  float* s_mx = reinterpret_cast<float*>(smem + kBOffMisc + kBMiscMx);      // [kBWg][128]
+  float* s_lp = reinterpret_cast<float*>(smem + kBOffMisc + kBMiscL);       // [kBWg][128], same memory
   uint32_t* status = reinterpret_cast<uint32_t*>(a.workspace);
   int* ws_pre = reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(a.workspace) + kWsHeaderBytes);
   float* ws_slots = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(a.workspace) + kWsHeaderBytes +
@@ -245,10 +248,10 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
     mbar_init(bars + 8 * kBbQEmpty, 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(bars + 8 * (kBbSFull + i), 1);
-      mbar_init(bars + 8 * (kBbPFull + i), 8);
+      mbar_init(bars + 8 * (kBbPFull + i), 4 * kBWg);
       mbar_init(bars + 8 * (kBbPvDone + i), 1);
     }
-    mbar_init(bars + 8 * kBbAll, 8);
+    mbar_init(bars + 8 * kBbAll, 4 * kBWg);
     mbar_init(bars + 8 * kBbDrain, 1);
     *abort_flag = 0;
     *grow_flag = 0;
@@ -383,7 +386,7 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
       }
     }
   } else if (warp >= 4 && n_iter > 0) {
-    // ====== softmax warps: thread = packed row; warpgroup g = key columns / output columns [64g, 64g+64) ======
+    // ====== softmax warps: thread = packed row; warpgroup g = key columns / output columns [kBCw*g, kBCw*(g+1)) ======
     const int wg = (warp - 4) >> 2, quad = (warp - 4) & 3;
     const int r = quad * 32 + lane;
     const uint32_t lane_addr = tmem + (static_cast<uint32_t>(quad * 32) << 16);
@@ -397,13 +400,19 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
     auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {
       return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, status));
     };
-    // bounded barrier of the eight softmax warps (also publishes their shared-memory writes)
-    auto sync8 = [&]() -> bool {
+    // bounded barrier of all softmax warps (also publishes their shared-memory writes)
+    auto sync_all = [&]() -> bool {
       __syncwarp();
       if (lane == 0) mbar_arrive(bars + 8 * kBbAll);
       const bool good = wait_all(bars + 8 * kBbAll, all_phase & 1);
       ++all_phase;
       return good;
+    };
+    auto max_of_groups = [&](const float* arr) -> float {
+      float m = arr[r];
+#pragma unroll
+      for (int g = 1; g < kBWg; ++g) m = fmaxf(m, arr[g * kTile + r]);
+      return m;
     };
     while (ok && w.it < n_iter) {
       bwalk_tile(w);
@@ -433,45 +442,43 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
         if (!wait_all(bars + 8 * (kBbKvFull + buf), (use / kBKv) & 1)) { ok = false; break; }
         const uint32_t va = sb + kBOffKv + buf * kBKvBytes;
         const int n_rows = ((nv + 15) & ~15) - nv;
-        for (int x = wg * 128 + r; x < n_rows * HALVES * 8; x += 256) {
+        for (int x = wg * kTile + r; x < n_rows * HALVES * 8; x += kBWg * kTile) {
           const int rr = nv + x / (HALVES * 8), cc = x % (HALVES * 8);
           const uint32_t addr = va + (cc >> 3) * kBHalf + rr * 128 + ((cc & 7) << 4);
           asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(addr), "r"(0u) : "memory");
         }
       }
-      // this warpgroup's 64 score columns of the row; invisible keys become -inf
-      const uint32_t s_addr = lane_addr + kBColS + pb * kTile + wg * 64;
-      const int key0 = (is_step ? w.step_idx * kTile : 0) + wg * 64;   // step-local index of column 0
-      float v[64];
-      auto load_scores = [&]() {
-        if (masked)
-          big_load_scores<true>(s_addr, v, wg * 64, nv, is_step, tok, key0, w.s.n_c, anc);
-        else
-          big_load_scores<false>(s_addr, v, 0, kTile, false, 0, 0, 0, 0);
-      };
-      load_scores();
+      // this warpgroup's score columns of the row; invisible keys become -inf
+      const uint32_t s_addr = lane_addr + kBColS + pb * kTile + wg * kBCw;
+      const int key0 = (is_step ? w.step_idx * kTile : 0) + wg * kBCw;   // step-local index of column 0
+      float v[kBCw];
+      if (masked)
+        big_load_scores<true>(s_addr, v, wg * kBCw, nv, is_step, tok, key0, w.s.n_c, anc);
+      else
+        big_load_scores<false>(s_addr, v, 0, kTile, false, 0, 0, 0, 0);
       if (w.piece_j == 0) {
-        // new unit: reference = exact maximum of the first tile over both column halves
-        s_mx[wg * 128 + r] = max64(v);
-        if (!sync8()) { ok = false; break; }
-        const float m = fmaxf(s_mx[r], s_mx[128 + r]);
+        // new unit: reference = exact maximum of the first tile over all column groups
+        s_mx[wg * kTile + r] = max_cols(v);
+        if (!sync_all()) { ok = false; break; }
+        const float m = max_of_groups(s_mx);
         m_ref = (m == -INFINITY) ? 0.f : m * a.scale_log2;
         l_part = 0.f;
       }
-      // p = 2^(s*scale - m_ref) as bf16 into this row of the P tile (half g = this group's 64 keys);
-      // returns the row's partial sum over those keys
-      const uint32_t p_row = sb + kBOffP + pb * kBPBytes + wg * kBHalf + r * 128;
+      // p = 2^(s*scale - m_ref) as bf16 into this row of the P tile; the row's partial sum over
+      // this group's keys
+      const uint32_t p_row = sb + kBOffP + pb * kBPBytes + ((wg * kBCw) >> 6) * kBHalf + r * 128;
+      const int chunk0 = ((wg * kBCw) & 63) >> 3;             // first 16-byte chunk inside the 64-key half
       auto p_pass = [&]() -> float {
         float ls[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {
+        for (int c = 0; c < kBCw / 8; ++c) {
           float p[8];
 #pragma unroll
           for (int e = 0; e < 8; ++e) {
             p[e] = ex2(fmaf(v[c * 8 + e], a.scale_log2, -m_ref));
             ls[e & 3] += p[e];
           }
-          const uint32_t addr = p_row + ((c ^ rx) << 4);
+          const uint32_t addr = p_row + (((chunk0 + c) ^ rx) << 4);
           asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(pack2(p[0], p[1])),
                        "r"(pack2(p[2], p[3])), "r"(pack2(p[4], p[5])), "r"(pack2(p[6], p[7]))
                        : "memory");
@@ -480,15 +487,15 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
       };
       float tsum = p_pass();
       // A score that outgrew the row reference by ~2^48 shows in the sum (so do inf and NaN); the
-      // eight warps agree on it before anyone hands P over
+      // softmax warps agree on it before anyone hands P over
       if (w.piece_j > 0 && __any_sync(0xffffffffu, row_ok && !(tsum < kBGrowSum)) && lane == 0)
         *grow_flag = it + 1;
-      if (!sync8()) { ok = false; break; }
+      if (!sync_all()) { ok = false; break; }
       if (*grow_flag == it + 1) {
-        // ---- rare: move the row references up; rescale O (this group's 64 columns) and the sums ----
-        s_mx[wg * 128 + r] = max64(v);
-        if (!sync8()) { ok = false; break; }
-        const float m = fmaxf(s_mx[r], s_mx[128 + r]);
+        // ---- rare: move the row references up; rescale O (this group's columns) and the sums ----
+        s_mx[wg * kTile + r] = max_cols(v);
+        if (!sync_all()) { ok = false; break; }
+        const float m = max_of_groups(s_mx);
         const float m_new = (m == -INFINITY) ? m_ref : fmaxf(m_ref, m * a.scale_log2);
         const float alpha = ex2(m_ref - m_new);
         m_ref = m_new;
@@ -496,17 +503,17 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
         if (!wait_all(bars + 8 * (kBbPvDone + ((it - 1) & 1)), ((it - 1) >> 1) & 1)) { ok = false; break; }
         tc_fence_after();
 #pragma unroll 1
-        for (int c = 0; c < 2; ++c) {
+        for (int c = 0; c < kBCw / 32; ++c) {
           uint32_t o[32];
-          tmem_ld32(lane_addr + kBColO + wg * 64 + c * 32, o);
+          tmem_ld32(lane_addr + kBColO + wg * kBCw + c * 32, o);
           tmem_ld_wait(o);
 #pragma unroll
           for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-          tmem_st32(lane_addr + kBColO + wg * 64 + c * 32, o);
+          tmem_st32(lane_addr + kBColO + wg * kBCw + c * 32, o);
         }
         asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
         tsum = p_pass();
-        if (!sync8()) { ok = false; break; }     // s_mx may be rewritten from here on
+        if (!sync_all()) { ok = false; break; }     // s_mx may be rewritten from here on
       }
       l_part += tsum;
       fence_async_smem();
@@ -515,10 +522,12 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
       if (lane == 0) mbar_arrive(bars + 8 * (kBbPFull + pb));
 
       if (w.last) {
-        // ---- end of the unit (or of this CTA's part of it) ----
-        s_lp[wg * 128 + r] = l_part;
-        if (!sync8()) { ok = false; break; }
-        const float l_row = s_lp[r] + s_lp[128 + r];
+        // ---- end of the item: the unit, or this chunk of it ----
+        s_lp[wg * kTile + r] = l_part;
+        if (!sync_all()) { ok = false; break; }
+        float l_row = 0.f;
+#pragma unroll
+        for (int g = 0; g < kBWg; ++g) l_row += s_lp[g * kTile + r];
         if (!wait_all(bars + 8 * (kBbPvDone + pb), (it >> 1) & 1)) { ok = false; break; }
         tc_fence_after();
         const int i = tok, g = r % a.G;
@@ -526,12 +535,12 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
         float* slot = ws_slots + static_cast<size_t>(w.slot < 0 ? 0 : w.slot) * big_slot_floats();
         const float inv = 1.f / l_row;
 #pragma unroll 1
-        for (int c = 0; c < 2; ++c) {
+        for (int c = 0; c < kBCw / 32; ++c) {
           uint32_t o[32];
-          tmem_ld32(lane_addr + kBColO + wg * 64 + c * 32, o);
+          tmem_ld32(lane_addr + kBColO + wg * kBCw + c * 32, o);
           tmem_ld_wait(o);
           if (row_ok && w.slot < 0) {
-            uint4* op = reinterpret_cast<uint4*>(a.out + orow * D + wg * 64 + c * 32);
+            uint4* op = reinterpret_cast<uint4*>(a.out + orow * D + wg * kBCw + c * 32);
 #pragma unroll
             for (int q4 = 0; q4 < 4; ++q4) {
               uint4 u;
@@ -542,7 +551,7 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
               op[q4] = u;
             }
           } else if (row_ok) {
-            uint4* sp = reinterpret_cast<uint4*>(slot + static_cast<size_t>(r) * D + wg * 64 + c * 32);
+            uint4* sp = reinterpret_cast<uint4*>(slot + static_cast<size_t>(r) * D + wg * kBCw + c * 32);
 #pragma unroll
             for (int q4 = 0; q4 < 8; ++q4) sp[q4] = make_uint4(o[4 * q4], o[4 * q4 + 1], o[4 * q4 + 2], o[4 * q4 + 3]);
           }
@@ -556,7 +565,8 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
             sm[kTile + r] = l_row;
           }
         }
-        tc_fence_before();   // the reads of O are ordered before the next unit's first PV product
+        tc_fence_before();   // the reads of O are ordered before the next item's first PV product
+        if (!sync_all()) { ok = false; break; }   // s_lp and s_mx share their memory with the next item
       }
       bwalk_next(a, w, pre);
     }
