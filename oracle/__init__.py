@@ -141,10 +141,15 @@ def rope(x: np.ndarray, pos_id: np.ndarray, rope_base: float, inv_freq=None, fla
     return x
 
 
+KIND_PROMPT, KIND_REASON, KIND_FORESIGHT, KIND_MEMORY, KIND_OUTPUT = 0, 1, 2, 3, 4
+
+
 def attn_step(k_cache, v_cache, kv_head_stride, kv_off, kv_len, q_off, n_cand, anchor,
-              q, k_step, v_step, sm_scale=None):
+              q, k_step, v_step, sm_scale=None, tok_kind=None, tok_step=None):
     """One layer of step attention.  k_cache/v_cache: uint16 flat or [H_kv][slots][D];
     q: uint16 [T][H_q][D]; k_step/v_step: uint16 [T][H_kv][D].
+    tok_kind (uint8 [T]) / tok_step (int32 [T]), both or neither: the block's own keys follow the
+    training-time mask of Sec. 2.3 (KIND_* below) instead of the (n_cand, anchor) rule.
     Returns (out fp64 [T][H_q][D], lse fp64 [T][H_q])."""
     q = np.ascontiguousarray(q, dtype=np.uint16)
     k_step = np.ascontiguousarray(k_step, dtype=np.uint16)
@@ -164,11 +169,14 @@ def attn_step(k_cache, v_cache, kv_head_stride, kv_off, kv_len, q_off, n_cand, a
         sm_scale = 1.0 / np.sqrt(float(D))
     out = np.empty((T, H_q, D), dtype=np.float64)
     lse = np.empty((T, H_q), dtype=np.float64)
-    rc = lib().ms_oracle_attn_step(
+    tk = None if tok_kind is None else np.ascontiguousarray(tok_kind, dtype=np.uint8)
+    ts = None if tok_step is None else np.ascontiguousarray(tok_step, dtype=np.int32)
+    assert (tk is None) == (ts is None)
+    rc = lib().ms_oracle_attn_block(
         C.c_int32(B), C.c_int32(H_q), C.c_int32(H_kv), C.c_int32(D),
         _p(k_cache, C.c_uint16), _p(v_cache, C.c_uint16), C.c_int64(kv_head_stride),
         _p(kv_off, C.c_int64), _p(kv_len, C.c_int32), _p(q_off, C.c_int32),
-        _p(n_cand, C.c_int32), _p(a, C.c_int32), _p(q, C.c_uint16), _p(k_step, C.c_uint16),
+        _p(n_cand, C.c_int32), _p(a, C.c_int32), _p(tk, C.c_uint8), _p(ts, C.c_int32), _p(q, C.c_uint16), _p(k_step, C.c_uint16),
         _p(v_step, C.c_uint16), C.c_double(sm_scale), _p(out, C.c_double), _p(lse, C.c_double))
     _chk(rc, "attn_step")
     return out, lse

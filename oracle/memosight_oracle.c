@@ -230,6 +230,25 @@ int32_t ms_oracle_visible(int32_t i, int32_t j, int32_t n_c, int32_t a_i) {
   return j < a_i;                  /* foresight: the candidates it follows */
 }
 
+/* Training-time mask over an augmented sequence (Sec. 2.3 "Attention Mask Strategy"): every
+ * token of the block carries a kind and the index of its reasoning step.  Key j of the block
+ * is visible to query i of the block iff it is the query itself, or it comes before the query
+ * and is not a foresight token (whose hidden state is masked from all later tokens) and is
+ * not a verbose reasoning token of another step (for previous steps only the prompt, memory
+ * and output tokens stay visible; inside the current step attention is causal). */
+#define MS_KIND_PROMPT 0
+#define MS_KIND_REASON 1
+#define MS_KIND_FORESIGHT 2
+#define MS_KIND_MEMORY 3
+#define MS_KIND_OUTPUT 4
+int32_t ms_oracle_visible_train(int32_t i, int32_t j, int32_t kind_j, int32_t step_i, int32_t step_j) {
+  if (j == i) return 1;
+  if (j > i) return 0;
+  if (kind_j == MS_KIND_FORESIGHT) return 0;
+  if (kind_j == MS_KIND_REASON) return step_j == step_i;
+  return 1;
+}
+
 /* ------------------------------------------------------------------------ */
 /* Step attention (definition of masked softmax attention, GQA)              */
 /* ------------------------------------------------------------------------ */
@@ -242,14 +261,23 @@ int32_t ms_oracle_visible(int32_t i, int32_t j, int32_t n_c, int32_t a_i) {
  * of candidates it sees; ignored for candidate rows.
  * Query head h reads KV head h / (H_q/H_kv).
  * out fp64 [T][H_q][D], lse fp64 [T][H_q] (natural log), either may be NULL. */
-int32_t ms_oracle_attn_step(int32_t B, int32_t H_q, int32_t H_kv, int32_t D,
-                            const uint16_t* k_cache, const uint16_t* v_cache,
-                            int64_t kv_head_stride, const int64_t* kv_off,
-                            const int32_t* kv_len, const int32_t* q_off,
-                            const int32_t* n_cand, const int32_t* anchor,
-                            const uint16_t* q, const uint16_t* k_step,
-                            const uint16_t* v_step, double sm_scale,
-                            double* out, double* lse) {
+static int32_t local_visible(int32_t i, int32_t j, int32_t n_c, int32_t a_i, int32_t r0,
+                             const uint8_t* tok_kind, const int32_t* tok_step) {
+  if (tok_kind) return ms_oracle_visible_train(i, j, tok_kind[r0 + j], tok_step[r0 + i], tok_step[r0 + j]);
+  return ms_oracle_visible(i, j, n_c, a_i);
+}
+
+/* tok_kind / tok_step [T] (both or neither): when given, the block's own keys follow the
+ * training-time rule above instead of the (n_cand, anchor) rule. */
+int32_t ms_oracle_attn_block(int32_t B, int32_t H_q, int32_t H_kv, int32_t D,
+                             const uint16_t* k_cache, const uint16_t* v_cache,
+                             int64_t kv_head_stride, const int64_t* kv_off,
+                             const int32_t* kv_len, const int32_t* q_off,
+                             const int32_t* n_cand, const int32_t* anchor,
+                             const uint8_t* tok_kind, const int32_t* tok_step,
+                             const uint16_t* q, const uint16_t* k_step,
+                             const uint16_t* v_step, double sm_scale,
+                             double* out, double* lse) {
   if (B < 0 || H_kv < 1 || H_q < 1 || H_q % H_kv || D < 1) return MS_ORACLE_BAD_ARG;
   const int32_t G = H_q / H_kv;
   int32_t bad = 0;
@@ -274,7 +302,7 @@ int32_t ms_oracle_attn_step(int32_t B, int32_t H_q, int32_t H_kv, int32_t D,
           if (j < L) {
             kv = Kc + (int64_t)j * D;
           } else {
-            if (!ms_oracle_visible(i, j - L, n_c, a_i)) { s[j] = -INFINITY; continue; }
+            if (!local_visible(i, j - L, n_c, a_i, r0, tok_kind, tok_step)) { s[j] = -INFINITY; continue; }
             kv = k_step + ((int64_t)(r0 + j - L) * H_kv + kvh) * D;
           }
           double dot = 0.0;
@@ -285,7 +313,7 @@ int32_t ms_oracle_attn_step(int32_t B, int32_t H_q, int32_t H_kv, int32_t D,
         /* softmax weights; a hidden key keeps weight exactly 0 */
         double denom = 0.0;
         for (int32_t j = 0; j < L + n_q; ++j) {
-          int32_t hidden = (j >= L) && !ms_oracle_visible(i, j - L, n_c, a_i);
+          int32_t hidden = (j >= L) && !local_visible(i, j - L, n_c, a_i, r0, tok_kind, tok_step);
           s[j] = hidden ? 0.0 : exp(s[j] - m);
           denom += s[j];
         }
@@ -293,7 +321,7 @@ int32_t ms_oracle_attn_step(int32_t B, int32_t H_q, int32_t H_kv, int32_t D,
           double* o = out + ((int64_t)(r0 + i) * H_q + h) * D;
           for (int32_t e = 0; e < D; ++e) o[e] = 0.0;
           for (int32_t j = 0; j < L + n_q; ++j) {
-            if ((j >= L) && !ms_oracle_visible(i, j - L, n_c, a_i)) continue;
+            if ((j >= L) && !local_visible(i, j - L, n_c, a_i, r0, tok_kind, tok_step)) continue;
             const uint16_t* vv = (j < L) ? Vc + (int64_t)j * D
                                          : v_step + ((int64_t)(r0 + j - L) * H_kv + kvh) * D;
             for (int32_t e = 0; e < D; ++e) o[e] += s[j] * bf16_to_f64(vv[e]);
@@ -306,6 +334,19 @@ int32_t ms_oracle_attn_step(int32_t B, int32_t H_q, int32_t H_kv, int32_t D,
     }
   }
   return bad ? MS_ORACLE_BAD_ARG : MS_ORACLE_OK;
+}
+
+/* The step block of inference: the (n_cand, anchor) rule for the block's own keys. */
+int32_t ms_oracle_attn_step(int32_t B, int32_t H_q, int32_t H_kv, int32_t D,
+                            const uint16_t* k_cache, const uint16_t* v_cache,
+                            int64_t kv_head_stride, const int64_t* kv_off,
+                            const int32_t* kv_len, const int32_t* q_off,
+                            const int32_t* n_cand, const int32_t* anchor,
+                            const uint16_t* q, const uint16_t* k_step,
+                            const uint16_t* v_step, double sm_scale,
+                            double* out, double* lse) {
+  return ms_oracle_attn_block(B, H_q, H_kv, D, k_cache, v_cache, kv_head_stride, kv_off, kv_len, q_off,
+                              n_cand, anchor, NULL, NULL, q, k_step, v_step, sm_scale, out, lse);
 }
 
 /* ------------------------------------------------------------------------ */
