@@ -158,7 +158,20 @@ typedef struct memosight_attn_params {
   size_t workspace_bytes;    /* >= memosight_attn_workspace_bytes(...)                         */
   void* ev_split_begin;      /* optional cudaEvent_t recorded on `stream` right before ...     */
   void* ev_split_end;        /* ... and right after the split-KV kernel (NULL: not recorded)   */
+  /* Optional training-time mask (Sec. 2.3 "Attention Mask Strategy"), both or neither.  The block
+   * is then an augmented sequence (Sec. 2.2) whose tokens carry a kind and a reasoning-step index;
+   * among the block's own keys, key j is visible to row i iff j == i, or j < i and j is neither a
+   * foresight token nor a reasoning token of another step.  n_cand and anchor are ignored.  A
+   * structure that ends before these fields (an older struct_size) means "not given". */
+  const uint8_t* tok_kind;   /* device [T]: MS_KIND_*                                          */
+  const int32_t* tok_step;   /* device [T]: index of the token's reasoning step (prompt: any)  */
 } memosight_attn_params;
+
+#define MS_KIND_PROMPT 0
+#define MS_KIND_REASON 1      /* a verbose reasoning token: visible inside its own step only    */
+#define MS_KIND_FORESIGHT 2   /* visible to itself only                                          */
+#define MS_KIND_MEMORY 3
+#define MS_KIND_OUTPUT 4
 
 /* Scratch size for memosight_attn_step with these bounds (0 on invalid input). */
 MS_API size_t memosight_attn_workspace_bytes(int32_t batch, int32_t n_q_heads, int32_t n_kv_heads,
@@ -171,8 +184,8 @@ MS_API size_t memosight_attn_workspace_bytes(int32_t batch, int32_t n_q_heads, i
  * forwards the ceil(n/c) memory tokens and <o> of a finished step as one causal block
  * (Sec. 2.1.2, Algorithm 1), and the prefill of a prompt is one causal block against an empty
  * or partly filled cache (Algorithm 1, Prefill) -- take the large-block tcgen05 kernel when D
- * is 128.  Anything
- * else inside the limits takes the slower general kernel.  Size the workspace with the very
+ * is 128; so do blocks with the training-time mask (tok_kind / tok_step) when max_nq > 16.
+ * Anything else inside the limits takes the slower general kernel.  Size the workspace with the very
  * batch, head counts, max_kv_len and max_nq of the call: a large-block call needs a different
  * amount than a step-block call.
  * The workspace may be reused by the next call on the same stream; two calls

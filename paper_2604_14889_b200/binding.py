@@ -32,6 +32,8 @@ MS_ATTN_PATH_TCGEN05 = 2
 MS_ATTN_PATH_GENERAL = 3
 MS_ATTN_PATH_TCGEN05_KEYS = 4
 
+MS_KIND_PROMPT, MS_KIND_REASON, MS_KIND_FORESIGHT, MS_KIND_MEMORY, MS_KIND_OUTPUT = 0, 1, 2, 3, 4
+
 MS_ROPE_NEOX = 0
 MS_ROPE_INTERLEAVED = 1
 MS_POS_HALF_UNITS = 2
@@ -63,6 +65,7 @@ class AttnParams(C.Structure):
         ("out", C.c_void_p), ("lse", C.c_void_p),
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
         ("ev_split_begin", C.c_void_p), ("ev_split_end", C.c_void_p),
+        ("tok_kind", C.c_void_p), ("tok_step", C.c_void_p),
     ]
 
 
@@ -254,7 +257,7 @@ def memosight_attn_workspace_bytes(batch: int, n_q_heads: int, n_kv_heads: int, 
 def attn_params(*, batch, n_q_heads, n_kv_heads, head_dim, k_cache, v_cache, kv_head_stride, n_slots,
                 kv_off, kv_len, max_kv_len, max_nq, q_off, n_cand, anchor, total_rows, sm_scale,
                 q, k_step, v_step, out, lse, workspace, workspace_bytes, ev_split_begin=None,
-                ev_split_end=None) -> AttnParams:
+                ev_split_end=None, tok_kind=None, tok_step=None) -> AttnParams:
     """Fills a memosight_attn_params structure (addresses only; nothing is copied)."""
     p = AttnParams()
     p.struct_size = C.sizeof(AttnParams)
@@ -269,6 +272,7 @@ def attn_params(*, batch, n_q_heads, n_kv_heads, head_dim, k_cache, v_cache, kv_
     p.out, p.lse = _ptr(out), _ptr(lse)
     p.workspace, p.workspace_bytes = _ptr(workspace), workspace_bytes
     p.ev_split_begin, p.ev_split_end = _ptr(ev_split_begin), _ptr(ev_split_end)
+    p.tok_kind, p.tok_step = _ptr(tok_kind), _ptr(tok_step)
     return p
 
 

@@ -1,6 +1,7 @@
 // Entry points of the step attention: argument validation, path selection,
 // workspace sizing and the device status word.
 #include <math.h>
+#include <stddef.h>
 
 #include "attn_internal.cuh"
 
@@ -63,7 +64,13 @@ extern "C" size_t memosight_attn_workspace_bytes(int32_t batch, int32_t n_q_head
 }
 
 extern "C" int32_t memosight_attn_step(const memosight_attn_params* p, memosight_stream_t stream) {
-  if (!p || p->struct_size != sizeof(memosight_attn_params)) return MS_ERR_INVALID_ARG;
+  // structures of callers built before the training-mask fields existed end at tok_kind
+  constexpr uint32_t kOldSize = offsetof(memosight_attn_params, tok_kind);
+  if (!p || (p->struct_size != sizeof(memosight_attn_params) && p->struct_size != kOldSize)) return MS_ERR_INVALID_ARG;
+  const bool has_meta = p->struct_size == sizeof(memosight_attn_params);
+  const uint8_t* tok_kind = has_meta ? p->tok_kind : nullptr;
+  const int32_t* tok_step = has_meta ? p->tok_step : nullptr;
+  if ((tok_kind == nullptr) != (tok_step == nullptr)) return MS_ERR_INVALID_ARG;
   if (p->batch < 0 || p->n_kv_heads < 1 || p->n_q_heads < 1 || p->head_dim < 1 ||
       p->max_kv_len < 0 || p->total_rows < 0 || p->n_slots < 0 || p->kv_head_stride < 0)
     return MS_ERR_INVALID_ARG;
@@ -97,6 +104,8 @@ extern "C" int32_t memosight_attn_step(const memosight_attn_params* p, memosight
   a.n_slots = p->n_slots;
   a.kv_off = p->kv_off; a.kv_len = p->kv_len; a.q_off = p->q_off; a.n_cand = p->n_cand;
   a.anchor = p->anchor;
+  a.tok_kind = tok_kind;
+  a.tok_step = tok_step;
   a.q = static_cast<const __nv_bfloat16*>(p->q);
   a.k_step = static_cast<const __nv_bfloat16*>(p->k_step);
   a.v_step = static_cast<const __nv_bfloat16*>(p->v_step);
@@ -112,8 +121,8 @@ extern "C" int32_t memosight_attn_step(const memosight_attn_params* p, memosight
 
   cudaStream_t st = ms::as_stream(stream);
   // An empty cache tensor still needs a valid address for the tile descriptors.
-  const int32_t path = (a.k_cache && a.v_cache && a.n_slots >= 1) ? pick_path(a.D, G, a.max_nq)
-                                                                   : MS_ATTN_PATH_GENERAL;
+  int32_t path = (a.k_cache && a.v_cache && a.n_slots >= 1) ? pick_path(a.D, G, a.max_nq) : MS_ATTN_PATH_GENERAL;
+  if (tok_kind && path != kPathBig) path = MS_ATTN_PATH_GENERAL;   // the step kernels know the inference rule only
   if (path == MS_ATTN_PATH_MMA_SYNC) return ms::launch_attn_mma(a, st);
   if (path == MS_ATTN_PATH_TCGEN05) return ms::launch_attn_umma(a, st);
   if (path == MS_ATTN_PATH_TCGEN05_KEYS) return ms::launch_attn_umma_t(a, st);

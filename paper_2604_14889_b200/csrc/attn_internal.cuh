@@ -19,6 +19,8 @@ struct AttnArgs {
   const int32_t* q_off;
   const int32_t* n_cand;
   const int32_t* anchor;
+  const uint8_t* tok_kind;    // training-time mask metadata, or NULL
+  const int32_t* tok_step;
   const __nv_bfloat16* q;
   const __nv_bfloat16* k_step;
   const __nv_bfloat16* v_step;
@@ -53,7 +55,7 @@ int32_t launch_attn_umma_t(const AttnArgs& a, cudaStream_t st);
 
 // tcgen05 path for large blocks (17..256 tokens per block, head_dim 128): the block is cut
 // into row tiles; own schedule, workspace size and merge kernel.
-bool attn_umma_big_supports(int D, int G, int max_nq);
+bool attn_umma_big_supports(int D, int G, int max_nq);   // the only tensor-core kernel that takes tok_kind/tok_step
 size_t attn_umma_big_workspace_bytes(int B, int H_kv, int G, int max_nq, int max_kv_len, int n_ctas);
 int32_t launch_attn_umma_big(const AttnArgs& a, cudaStream_t st);
 

@@ -47,7 +47,9 @@ attn_simt_kernel(AttnArgs a) {
       vp = Vc + static_cast<int64_t>(j) * D;
     } else {
       const int jj = j - L;
-      if (!step_key_visible(i, jj, n_c, a_i)) continue;   // warp-uniform
+      const bool vis = a.tok_kind ? train_key_visible(i, jj, a.tok_kind[r0 + jj], a.tok_step[t], a.tok_step[r0 + jj])
+                                  : step_key_visible(i, jj, n_c, a_i);
+      if (!vis) continue;                                  // warp-uniform
       kp = a.k_step + (static_cast<int64_t>(r0 + jj) * a.H_kv + kvh) * D;
       vp = a.v_step + (static_cast<int64_t>(r0 + jj) * a.H_kv + kvh) * D;
     }

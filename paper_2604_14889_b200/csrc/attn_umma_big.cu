@@ -172,9 +172,13 @@ __device__ __host__ inline size_t big_slot_floats() { return static_cast<size_t>
 // The warpgroup's 64 score columns of one row, from tensor memory into v[]; with kMasked the
 // invisible keys (past the valid length; on a step-local tile by the (n_cand, anchor) rule)
 // become -inf.
+// (With meta_kind the step-local rule is the training-time one: kind/step of key token j at
+// meta_kind[j] / meta_step[j], the row's own step in anc.)
 template <bool kMasked>
 __device__ __forceinline__ void big_load_scores(uint32_t s_addr, float (&v)[kBCw], int col0, int nv, bool is_step,
-                                                int tok, int key0, int n_c, int anc) {
+                                                int tok, int key0, int n_c, int anc,
+                                                const uint8_t* __restrict__ meta_kind = nullptr,
+                                                const int32_t* __restrict__ meta_step = nullptr) {
   uint32_t raw[kBCw / 32][32];
 #pragma unroll
   for (int c = 0; c < kBCw / 32; ++c) tmem_ld32(s_addr + c * 32, raw[c]);
@@ -185,7 +189,11 @@ __device__ __forceinline__ void big_load_scores(uint32_t s_addr, float (&v)[kBCw
     float s = __uint_as_float(raw[e >> 5][e & 31]);
     if (kMasked) {
       bool vis = col0 + e < nv;
-      if (is_step) vis = vis && step_key_visible(tok, key0 + e, n_c, anc);
+      if (is_step && vis) {
+        const int j = key0 + e;
+        vis = meta_kind ? train_key_visible(tok, j, __ldg(meta_kind + j), anc, __ldg(meta_step + j))
+                        : step_key_visible(tok, j, n_c, anc);
+      }
       s = vis ? s : -INFINITY;
     }
     v[e] = s;
@@ -424,7 +432,8 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
         if (row_ok) {
           const int i = tok0 + r / a.G;
           tok = i;
-          anc = (i < w.s.n_c) ? i : (a.anchor ? a.anchor[w.s.r0 + i] : w.s.n_c);
+          anc = a.tok_kind ? a.tok_step[w.s.r0 + i]            // training-time mask: the row's own step
+                           : ((i < w.s.n_c) ? i : (a.anchor ? a.anchor[w.s.r0 + i] : w.s.n_c));
         } else {
           tok = 1 << 20;
           anc = 0;
@@ -453,7 +462,8 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
       const int key0 = (is_step ? w.step_idx * kTile : 0) + wg * kBCw;   // step-local index of column 0
       float v[kBCw];
       if (masked)
-        big_load_scores<true>(s_addr, v, wg * kBCw, nv, is_step, tok, key0, w.s.n_c, anc);
+        big_load_scores<true>(s_addr, v, wg * kBCw, nv, is_step, tok, key0, w.s.n_c, anc,
+                              a.tok_kind ? a.tok_kind + w.s.r0 : nullptr, a.tok_kind ? a.tok_step + w.s.r0 : nullptr);
       else
         big_load_scores<false>(s_addr, v, 0, kTile, false, 0, 0, 0, 0);
       if (w.piece_j == 0) {

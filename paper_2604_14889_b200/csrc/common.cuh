@@ -44,4 +44,10 @@ __host__ __device__ inline bool step_key_visible(int i, int j, int n_c, int a_i)
   return (j == i) || (j < n_c && j < a_i);
 }
 
+// Training-time visibility among the block's own tokens (see memosight_attn_params::tok_kind).
+__host__ __device__ inline bool train_key_visible(int i, int j, int kind_j, int step_i, int step_j) {
+  return (j == i) ||
+         (j < i && kind_j != MS_KIND_FORESIGHT && (kind_j != MS_KIND_REASON || step_j == step_i));
+}
+
 }  // namespace ms
