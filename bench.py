@@ -459,7 +459,7 @@ def run_compress(args, ms, dev, world, rank):
     roofline is the bf16 tensor peak."""
     assert world == 1, "the compress workload is a single-GPU measurement"
     K, W = args.steps, max(args.warmup, 3)
-    B = args.batch if args.batch != 128 else 16
+    B = args.batch if args.batch != 128 else 64
     L0, nq, Hq, Hkv, D = args.kv_len, MEM_TOKENS + 1, 32, 8, 128
     growth = (K + W) * nq + SEG_LEN + 64
     cfg = synth.StepConfig("compress", B, Hq, Hkv, D, L0, L0, nq, 0, 5.0e5, 1024, headroom=growth, seed=0x5EED0004)

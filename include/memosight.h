@@ -194,10 +194,11 @@ MS_API int32_t memosight_attn_step(const memosight_attn_params* params, memosigh
 
 /* Diagnostic switch: which kernel memosight_attn_step uses from now on, process-wide.
  * MS_ATTN_PATH_AUTO (the default) picks by shape: head_dim 128 with up to 64 packed rows
- * (max_nq * H_q/H_kv) takes the keys-on-lanes tcgen05 kernel, 65..128 rows the rows-on-lanes
- * tcgen05 kernel, head_dim 64 the mma.sync kernel (up to 64 rows), anything else the general
- * kernel.  Forcing a path that does not cover a shape falls back to the automatic choice for
- * that call.  Returns the previous setting, or MS_ERR_INVALID_ARG.  Results of all paths agree
+ * (max_nq * H_q/H_kv) takes the keys-on-lanes tcgen05 kernel, more rows or blocks of more than
+ * 16 tokens the row-tiled large-block kernel; head_dim 64 the mma.sync kernel (up to 64 rows)
+ * or the rows-on-lanes tcgen05 kernel (up to 128); anything else the general kernel.  Forcing a path that does not cover a shape falls back to the automatic choice for
+ * that call (MS_ATTN_PATH_LARGE_BLOCK on a step block also needs a workspace of the size a
+ * large-block call of the same bounds would get).  Returns the previous setting, or MS_ERR_INVALID_ARG.  Results of all paths agree
  * within the tolerance of bf16 inputs with fp32 accumulation; the switch exists for tests and
  * timing. */
 #define MS_ATTN_PATH_AUTO 0
@@ -205,6 +206,7 @@ MS_API int32_t memosight_attn_step(const memosight_attn_params* params, memosigh
 #define MS_ATTN_PATH_TCGEN05 2
 #define MS_ATTN_PATH_GENERAL 3
 #define MS_ATTN_PATH_TCGEN05_KEYS 4   /* tcgen05 with the keys on the accumulator lanes; <= 64 rows, D 128 */
+#define MS_ATTN_PATH_LARGE_BLOCK 5    /* the row-tiled tcgen05 kernel of large blocks, for any block size; D 128 */
 MS_API int32_t memosight_attn_set_path(int32_t path);
 
 /* Synchronises `stream` and returns MS_OK, or MS_ERR_DEVICE_TIMEOUT if a kernel

@@ -31,6 +31,7 @@ MS_ATTN_PATH_MMA_SYNC = 1
 MS_ATTN_PATH_TCGEN05 = 2
 MS_ATTN_PATH_GENERAL = 3
 MS_ATTN_PATH_TCGEN05_KEYS = 4
+MS_ATTN_PATH_LARGE_BLOCK = 5
 
 MS_KIND_PROMPT, MS_KIND_REASON, MS_KIND_FORESIGHT, MS_KIND_MEMORY, MS_KIND_OUTPUT = 0, 1, 2, 3, 4
 

@@ -23,8 +23,9 @@ bool fast_path_shape(int D, int G, int max_nq) {
 
 // Which kernel serves a shape.  head_dim 128 with up to 64 packed rows -- every step block of
 // the method -- streams fastest through the keys-on-lanes tcgen05 kernel, whose softmax cost
-// follows the block size; 65..128 rows take the rows-on-lanes tcgen05 kernel; head_dim 64
-// stays on the mma.sync kernel up to 64 rows.
+// follows the block size; more rows or more than 16 tokens take the row-tiled large-block
+// kernel; head_dim 64 stays on the mma.sync kernel up to 64 rows and on the rows-on-lanes
+// tcgen05 kernel up to 128.
 int32_t pick_path(int D, int G, int max_nq) {
   const int32_t forced = g_forced_path.load(std::memory_order_relaxed);
   const bool mma_ok = mma_shape(D, G, max_nq), umma_ok = ms::attn_umma_supports(D, G, max_nq);
@@ -43,7 +44,7 @@ int32_t pick_path(int D, int G, int max_nq) {
 }  // namespace
 
 extern "C" int32_t memosight_attn_set_path(int32_t path) {
-  if (path < MS_ATTN_PATH_AUTO || path > MS_ATTN_PATH_TCGEN05_KEYS) return MS_ERR_INVALID_ARG;
+  if (path < MS_ATTN_PATH_AUTO || path > MS_ATTN_PATH_LARGE_BLOCK) return MS_ERR_INVALID_ARG;
   return g_forced_path.exchange(path, std::memory_order_relaxed);
 }
 
@@ -123,6 +124,11 @@ extern "C" int32_t memosight_attn_step(const memosight_attn_params* p, memosight
   // An empty cache tensor still needs a valid address for the tile descriptors.
   int32_t path = (a.k_cache && a.v_cache && a.n_slots >= 1) ? pick_path(a.D, G, a.max_nq) : MS_ATTN_PATH_GENERAL;
   if (tok_kind && path != kPathBig) path = MS_ATTN_PATH_GENERAL;   // the step kernels know the inference rule only
+  // the large-block kernel on a step block, when asked for and the workspace is large enough for it
+  if (g_forced_path.load(std::memory_order_relaxed) == MS_ATTN_PATH_LARGE_BLOCK && a.D == 128 && a.k_cache &&
+      a.v_cache && a.n_slots >= 1 &&
+      p->workspace_bytes >= ms::attn_umma_big_workspace_bytes(a.B, a.H_kv, G, a.max_nq, a.max_kv_len, ms::attn_mma_grid()))
+    path = kPathBig;
   if (path == MS_ATTN_PATH_MMA_SYNC) return ms::launch_attn_mma(a, st);
   if (path == MS_ATTN_PATH_TCGEN05) return ms::launch_attn_umma(a, st);
   if (path == MS_ATTN_PATH_TCGEN05_KEYS) return ms::launch_attn_umma_t(a, st);

@@ -669,8 +669,10 @@ int big_nsplit(int B, int H_kv, int max_rt, int n_ctas, int max_kv_len) {
 
 }  // namespace
 
+// Large blocks, and step blocks with more than 64 packed rows (where two softmax warpgroups per
+// tile beat the one of the rows-on-lanes step kernel: 5.2 against 4.2 TB/s at 128 rows).
 bool attn_umma_big_supports(int D, int G, int max_nq) {
-  return D == kBD && G >= 1 && G <= kMaxGroup && max_nq > kMaxNq && max_nq <= kMaxNqBig;
+  return D == kBD && G >= 1 && G <= kMaxGroup && max_nq <= kMaxNqBig && (max_nq > kMaxNq || G * max_nq > 64);
 }
 
 size_t attn_umma_big_workspace_bytes(int B, int H_kv, int G, int max_nq, int max_kv_len, int n_ctas) {
@@ -682,7 +684,7 @@ size_t attn_umma_big_workspace_bytes(int B, int H_kv, int G, int max_nq, int max
 
 int32_t launch_attn_umma_big(const AttnArgs& a, cudaStream_t st) {
   if (a.B == 0 || a.T == 0) return MS_OK;
-  if (!attn_umma_big_supports(a.D, a.G, a.max_nq)) return MS_ERR_UNSUPPORTED_SHAPE;
+  if (a.D != kBD || a.G > kMaxGroup || a.max_nq > kMaxNqBig) return MS_ERR_UNSUPPORTED_SHAPE;
   const int tpt = kTile / a.G;                   // tokens per row tile
   const int max_rt = (a.max_nq + tpt - 1) / tpt;
   const int grid = attn_mma_grid();
