@@ -49,7 +49,7 @@ __device__ __forceinline__ double bf16_bits_to_f64(uint16_t h) {
 
 __global__ void __launch_bounds__(128)
 rope_qk_kernel(uint16_t* __restrict__ q, uint16_t* __restrict__ k, const int32_t* __restrict__ pos_id,
-               int H_q, int H_kv, int D, uint32_t flags, FreqTable freq) {
+               int H_q, int H_kv, int D, uint32_t flags, bool vec_ok, FreqTable freq) {
   __shared__ double s_cos[kMaxHalf];
   __shared__ double s_sin[kMaxHalf];
   const int t = blockIdx.x;
@@ -65,6 +65,47 @@ rope_qk_kernel(uint16_t* __restrict__ q, uint16_t* __restrict__ k, const int32_t
   __syncthreads();
   const bool interleaved = (flags & MS_ROPE_INTERLEAVED) != 0;
   const int n_heads = H_q + H_kv;
+  if (vec_ok && (half & 7) == 0) {
+    // 16-byte accesses: a work item is 8 consecutive pair indices of one head (rotate-half: 8
+    // elements of each half) or 4 of them (interleaved: 8 consecutive elements)
+    const int per_head = interleaved ? half / 4 : half / 8;
+    for (int w = threadIdx.x; w < n_heads * per_head; w += blockDim.x) {
+      const int h = w / per_head, c = w - h * per_head;
+      uint16_t* v = (h < H_q) ? q + (static_cast<int64_t>(t) * H_q + h) * D
+                              : k + (static_cast<int64_t>(t) * H_kv + (h - H_q)) * D;
+      if (interleaved) {
+        uint4* p = reinterpret_cast<uint4*>(v + 8 * c);
+        uint4 x = *p;
+        uint16_t* e = reinterpret_cast<uint16_t*>(&x);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int i = 4 * c + j;
+          const double a = bf16_bits_to_f64(e[2 * j]), b = bf16_bits_to_f64(e[2 * j + 1]);
+          const double cs = s_cos[i], sn = s_sin[i];
+          e[2 * j] = f64_to_bf16_bits(a * cs - b * sn);
+          e[2 * j + 1] = f64_to_bf16_bits(b * cs + a * sn);
+        }
+        *p = x;
+      } else {
+        uint4* pa = reinterpret_cast<uint4*>(v + 8 * c);
+        uint4* pb = reinterpret_cast<uint4*>(v + half + 8 * c);
+        uint4 xa = *pa, xb = *pb;
+        uint16_t* ea = reinterpret_cast<uint16_t*>(&xa);
+        uint16_t* eb = reinterpret_cast<uint16_t*>(&xb);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int i = 8 * c + j;
+          const double a = bf16_bits_to_f64(ea[j]), b = bf16_bits_to_f64(eb[j]);
+          const double cs = s_cos[i], sn = s_sin[i];
+          ea[j] = f64_to_bf16_bits(a * cs - b * sn);
+          eb[j] = f64_to_bf16_bits(b * cs + a * sn);
+        }
+        *pa = xa;
+        *pb = xb;
+      }
+    }
+    return;
+  }
   for (int w = threadIdx.x; w < n_heads * half; w += blockDim.x) {
     const int h = w / half, i = w - h * half;
     uint16_t* v = (h < H_q) ? q + (static_cast<int64_t>(t) * H_q + h) * D
@@ -94,9 +135,10 @@ extern "C" int32_t memosight_rope_qk(void* q, void* k, const int32_t* pos_id, in
   for (int i = 0; i < D / 2; ++i)
     freq.f[i] = inv_freq ? inv_freq[i] : pow(rope_base, -2.0 * static_cast<double>(i) / D);
   for (int i = D / 2; i < kMaxHalf; ++i) freq.f[i] = 0.0;
+  const bool vec_ok = ms::aligned16(q) && ms::aligned16(k);   // NULL (no heads of that kind) counts as aligned
   rope_qk_kernel<<<T, 128, 0, ms::as_stream(stream)>>>(static_cast<uint16_t*>(q),
                                                         static_cast<uint16_t*>(k), pos_id, H_q, H_kv,
-                                                        D, flags, freq);
+                                                        D, flags, vec_ok, freq);
   MS_LAUNCH_CHECK();
   return MS_OK;
 }
