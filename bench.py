@@ -64,6 +64,15 @@ def parse_args():
     ap.add_argument("--workload", default="step", choices=["step", "compress"],
                     help="step: the Predict+Verify step the headline metric is quoted on (default); "
                          "compress: the compression event (forward of the memory tokens + <o>, append, eviction)")
+    ap.add_argument("--sweep", action="store_true",
+                    help="the foresight/batch/cache-length sweep (8B shape): one device-resident run per point, "
+                         "a table of KV bytes read, step tokens/s and HBM fraction on stdout")
+    ap.add_argument("--graph", action="store_true",
+                    help="after the timed region, also capture K further steps in one CUDA graph and time its "
+                         "replay (adds a \"graph\" object; needs --no-e2e)")
+    ap.add_argument("--uncompressed", action="store_true",
+                    help="the cache is an uncompressed one (position IDs = cache indices); with --kv-len 49152 "
+                         "it is the counterpart of the compacted 16K cache")
     ap.add_argument("--attn-path", default="auto", choices=["auto", "mma_sync", "tcgen05", "tcgen05_keys"],
                     help="attention kernel: by shape (default), or forced for A/B timing")
     return ap.parse_args()
@@ -86,9 +95,10 @@ def peak_hbm():
 
 class Schedule:
     """Host-side replay of what the step loop does to the cache lengths: the
-    synthetic drafts fix every sequence's accepted count, and one sequence per
-    step (round-robin) ends a 512-token reasoning step and is compacted.  Gives
-    the algorithmic bytes of each step and the compaction requests."""
+    synthetic drafts fix every sequence's accepted count, and every sequence ends
+    a 512-token reasoning step and is compacted once per 128 steps (round-robin:
+    one sequence per step at batch 128).  Gives the algorithmic bytes of each
+    step and the compaction requests."""
 
     def __init__(self, cfg, lens0, n_steps):
         B = cfg.batch
@@ -102,8 +112,8 @@ class Schedule:
             self.len_at.append(list(lens))
             for b in range(B):
                 lens[b] += self.keep[b]
-            b = s % B
-            if lens[b] >= SEG_LEN + tail:
+            b = s % max(B, 128)
+            if b < B and lens[b] >= SEG_LEN + tail:
                 self.seg_start[s, b] = lens[b] - tail - SEG_LEN
                 self.seg_len[s, b] = SEG_LEN
                 lens[b] -= SEG_LEN
@@ -257,10 +267,14 @@ def run_reference(args):
 
 def workload_config(cfg, args):
     return {"workload": f"8B-shape attention layer H_q={cfg.n_q_heads} H_kv={cfg.n_kv_heads} D={cfg.head_dim}, "
-                        f"batch {cfg.batch} per GPU, compacted KV {cfg.len_lo} per sequence, "
+                        f"batch {cfg.batch} per GPU, {'uncompressed' if args.uncompressed else 'compacted'} KV {cfg.len_lo} "
+                        f"per sequence, "
                         f"{cfg.n_cand} candidate + d={cfg.d} foresight rows per block, vocab {cfg.vocab}, 1 layer",
             "global_batch": cfg.batch * args.gpus, "kv_len": cfg.len_lo, "n_cand": cfg.n_cand, "d": cfg.d,
-            "l2": "per-step inputs (KV cache of several GB, logits) are far larger than the 126 MB L2; no flush",
+            "l2": ("per-step inputs (KV cache of several GB, logits) are far larger than the 126 MB L2; no flush"
+                   if cfg.batch * cfg.len_lo * cfg.n_kv_heads * cfg.head_dim * 4 > 4 * 126e6 else
+                   "the KV cache of this point is not much larger than the 126 MB L2: its bandwidth figure is "
+                   "not an HBM figure"),
             "parallelism": f"dp{args.gpus} (independent replicas by sequence, no collective on the data path)"}
 
 
@@ -280,8 +294,41 @@ def whole_job_throughput(units_per_rank: int, elapsed_ms_local: float, world: in
 
 # --------------------------------------------------------------------------- our arm
 
+def run_sweep(args):
+    """Runs this script once per sweep point (fresh process each: the caches are up to 26 GB) and
+    prints one table row per point plus the JSON lines."""
+    import subprocess
+    rows, lines = [], []
+    print("| d | batch | cache | KV GB/step | step ms | step ms (CUDA graph) | attention µs | step tokens/s | "
+          "step tokens/s (CUDA graph) | attention GB/s | of measured HBM | of 8 TB/s |")
+    print("|---:|---:|---|---:|---:|---:|---:|---:|---:|---:|---:|---:|", flush=True)
+    for kv_len, unc in ((16384, False), (49152, True)):
+        for d in range(1, 8):
+            for batch in (1, 8, 32, 128):
+                cmd = [sys.executable, os.path.abspath(__file__), "--batch", str(batch), "--d", str(d), "--kv-len",
+                       str(kv_len), "--steps", str(args.steps if args.steps != 200 else 30), "--warmup", "3",
+                       "--no-e2e", "--no-cpu-baseline", "--graph"] + (["--uncompressed"] if unc else [])
+                out = subprocess.run(cmd, capture_output=True, text=True)
+                if out.returncode != 0:
+                    print(out.stderr[-2000:], file=sys.stderr)
+                    raise SystemExit(out.returncode)
+                j = json.loads(out.stdout.strip().splitlines()[-1])
+                lines.append(j)
+                r = j["roofline"]
+                print(f"| {d} | {batch} | {'48K uncompressed' if unc else '16K compacted'} | {j['kv_gb_per_step']:.3f} | "
+                      f"{j['ms_per_step']:.3f} | {j['graph']['ms_per_step']:.3f} | {r['avg_launch_ms'] * 1e3:.1f} | "
+                      f"{j['value']:.0f} | {j['graph']['value']:.0f} | {r['achieved']:.0f} | "
+                      f"{r['frac']:.2f}{' (L2)' if j['kv_gb_per_step'] < 0.5 else ''} | {r['frac_of_nominal_8000']:.2f} |",
+                      flush=True)
+    for j in lines:
+        print(json.dumps(j))
+
+
 def main():
     args = parse_args()
+    if args.sweep:
+        run_sweep(args)
+        return
     if args.impl == "reference":
         run_reference(args)
         return
@@ -304,10 +351,12 @@ def main():
         run_compress(args, ms, dev, world, rank)
         return
     K, W = args.steps, max(args.warmup, 3)
-    cfg0 = synth.sweep(args.batch, args.d, args.kv_len, True)
+    cfg0 = synth.sweep(args.batch, args.d, args.kv_len, not args.uncompressed)
     n_e2e = 0 if args.no_e2e else max(1, min(args.e2e_steps, K))
     n_total = W + K
-    n_sched = n_total + (3 + n_e2e if n_e2e else 0)
+    if args.graph and n_e2e:
+        raise SystemExit("--graph needs --no-e2e")
+    n_sched = n_total + (3 + n_e2e if n_e2e else 0) + (K + 1 if args.graph else 0)
     growth = 3 * n_sched + SEG_LEN + 64
     cfg = synth.StepConfig(cfg0.name, cfg0.batch, cfg0.n_q_heads, cfg0.n_kv_heads, cfg0.head_dim, cfg0.len_lo,
                            cfg0.len_hi, cfg0.n_cand, cfg0.d, cfg0.rope_base, cfg0.vocab, headroom=growth,
@@ -390,6 +439,27 @@ def main():
 
     value, elapsed_ms = whole_job_throughput(T * K, elapsed_ms, world, dev)
 
+    graph_info = None
+    if args.graph:
+        # the same K-step loop as one CUDA graph: what the step costs once the host's launch work is gone
+        side = torch.cuda.Stream()
+        g = torch.cuda.CUDAGraph()
+        torch.cuda.synchronize()
+        with torch.cuda.graph(g, stream=side):
+            for s in range(K):
+                step(n_total + s)
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        g0.record()
+        g.replay()
+        g1.record()
+        barrier()
+        assert ms.memosight_attn_status(ws) == ms.MS_OK
+        assert inp.kv_len.cpu().tolist() == sched.len_at[n_total + K], "graph replay: cache lengths differ"
+        g_value, g_ms = whole_job_throughput(T * K, g0.elapsed_time(g1), world, dev)
+        graph_info = {"ms_per_step": g_ms / K, "value": g_value, "unit": UNIT,
+                      "note": "K further steps captured once in a CUDA graph, one replay timed"}
+
     # roofline of the dominant kernel (split-KV attention): algorithmic KV bytes per launch / its duration
     kv_bytes = [sched.kv_bytes(W + s, cfg) for s in range(K)]
     step_local = T * (2 * Hq + 2 * Hkv) * D * 2
@@ -429,6 +499,8 @@ def main():
     }
     if e2e is not None:
         line["e2e"] = e2e
+    if graph_info is not None:
+        line["graph"] = graph_info
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
             del inp, acc
