@@ -52,18 +52,26 @@ def test_schedule_replay_is_consistent():
     sys.path.insert(0, ROOT)
     import bench
     from paper_2604_14889_b200 import synth
-    cfg = synth.sweep(8, 3, 4096, True)
-    sch = bench.Schedule(cfg, [4096] * 8, 40)
-    assert all(1 <= k <= 3 for k in sch.keep)
-    lens = [4096] * 8
-    for s in range(40):
-        assert sch.len_at[s] == lens
-        lens = [l + k for l, k in zip(lens, sch.keep)]
-        b = s % 8
-        assert sch.seg_len[s].sum() == sch.seg_len[s, b] == 512
-        assert sch.seg_start[s, b] == lens[b] - 171 - 512
-        lens[b] -= 512
-    assert sch.final == lens
+    # every sequence is compacted once per 128 steps: one per step at batch 128, one step in 16 at batch 8
+    for B, n_steps in ((8, 300), (128, 140), (200, 210)):
+        cfg = synth.sweep(B, 3, 4096, True)
+        sch = bench.Schedule(cfg, [4096] * B, n_steps)
+        assert all(1 <= k <= 3 for k in sch.keep)
+        lens = [4096] * B
+        events = 0
+        for s in range(n_steps):
+            assert sch.len_at[s] == lens
+            lens = [l + k for l, k in zip(lens, sch.keep)]
+            b = s % max(B, 128)
+            if b < B:
+                assert sch.seg_len[s].sum() == sch.seg_len[s, b] == 512
+                assert sch.seg_start[s, b] == lens[b] - 171 - 512
+                lens[b] -= 512
+                events += 1
+            else:
+                assert sch.seg_len[s].sum() == 0
+        assert events == sum(1 for s in range(n_steps) if s % max(B, 128) < B)
+        assert sch.final == lens
 
 
 def test_reference_arm_other_ranks_exit_quietly():
