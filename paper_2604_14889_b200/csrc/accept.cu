@@ -2,9 +2,13 @@
 // logits, then per sequence the longest draft prefix equal to the argmax.
 //
 // The logits are read exactly once (HBM-bound).  Pass 1 cuts every row into
-// chunks so that small batches still fill the machine: one CTA per (chunk, row)
-// streams its chunk with 16-byte loads (8 in flight per thread) and leaves one
-// (value, index) candidate in the workspace.  Pass 2 uses one warp per sequence:
+// chunks of 8192 floats so that small batches still fill the machine and leaves one
+// (value, index) candidate per (row, chunk) in the workspace.  Its streaming form
+// (16-byte-aligned rows, vocabulary a multiple of 4) is one persistent CTA per SM:
+// a producer thread keeps six 32 KB bulk copies (cp.async.bulk, global -> shared
+// memory, completion on an mbarrier) in flight, six warps take a chunk each from
+// the ring and reduce it with shuffles only.  Other layouts fall back to one CTA per
+// (chunk, row) with plain loads.  Pass 2 uses one warp per sequence:
 // each lane folds the chunk candidates of one row, then lane 0 walks the block's
 // rows to count the matching prefix.  Ordering rule everywhere: a NaN beats any
 // number, larger value beats smaller, equal values (and two NaNs) go to the lower
@@ -13,6 +17,7 @@
 
 #include <mutex>
 
+#include "attn_sched.cuh"
 #include "common.cuh"
 
 namespace {
@@ -94,6 +99,136 @@ argmax_chunks_kernel(const float* __restrict__ logits, int64_t ld_v, int V, int 
   }
 }
 
+// ---- pass 1, streaming form -------------------------------------------------------------------
+
+constexpr int kStages = 6;                       // 32 KB chunks in flight per SM
+constexpr int kStreamWarps = kStages;             // warp w owns stage w: it follows that stage's barrier phase by phase
+constexpr int kStreamThreads = (kStreamWarps + 1) * 32;
+constexpr int kStageBytes = kChunk * 4;
+constexpr int kStreamSmem = kStages * kStageBytes + 2 * kStages * 8 + 16;
+
+// Set (to a magic word) if a wait inside the streaming kernel ever ran into its time limit; the
+// candidates of the chunks that were not finished then carry index -1, which matches no draft.
+static __device__ unsigned int g_accept_wait_status;
+
+__global__ void __launch_bounds__(kStreamThreads, 1)
+argmax_stream_kernel(const float* __restrict__ logits, int64_t ld_v, int V, int n_chunks, int n_items,
+                     Cand* __restrict__ part) {
+  extern __shared__ __align__(1024) uint8_t smem[];
+  const uint32_t sb = ms::smem_u32(smem);
+  const uint32_t bars = sb + kStages * kStageBytes;           // full[kStages], empty[kStages]
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kStages * kStageBytes + 2 * kStages * 8);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kStages; ++i) {
+      ms::mbar_init(bars + 8 * i, 1);
+      ms::mbar_init(bars + 8 * (kStages + i), 1);
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  // this CTA's items: blockIdx.x, blockIdx.x + gridDim.x, ...  (item = row * n_chunks + chunk)
+  const int n_local = (n_items - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) /
+                      static_cast<int>(gridDim.x);
+  if (warp == kStreamWarps) {
+    if (lane == 0) {
+      // ---- producer: one bulk copy per item into the ring
+      int issued = 0;
+      for (int k = 0; k < n_local; ++k) {
+        const int s = k % kStages;
+        if (!ms::mbar_wait(bars + 8 * (kStages + s), ((k / kStages) & 1) ^ 1, abort_flag, &g_accept_wait_status)) break;
+        const int item = static_cast<int>(blockIdx.x) + k * static_cast<int>(gridDim.x);
+        const int row = item / n_chunks, chunk = item - row * n_chunks;
+        const int lo = chunk * kChunk;
+        const uint32_t bytes = static_cast<uint32_t>(min(V, lo + kChunk) - lo) * 4u;
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the warps' reads of this stage come first
+        ms::mbar_arrive_expect_tx(bars + 8 * s, bytes);
+        asm volatile(
+            "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+            ::"r"(sb + s * kStageBytes), "l"(logits + static_cast<int64_t>(row) * ld_v + lo), "r"(bytes),
+              "r"(bars + 8 * s)
+            : "memory");
+        ++issued;
+      }
+      // copies still in flight must land before the CTA's shared memory goes away
+      for (int k = issued > kStages ? issued - kStages : 0; k < issued; ++k)
+        (void)ms::mbar_wait(bars + 8 * (k % kStages), (k / kStages) & 1, abort_flag, &g_accept_wait_status);
+    }
+    return;
+  }
+  // ---- consumers: warp w takes the items k = w, w + kStages, ... of this CTA (always stage w)
+  for (int k = warp; k < n_local; k += kStreamWarps) {
+    const int s = k % kStages;
+    const int item = static_cast<int>(blockIdx.x) + k * static_cast<int>(gridDim.x);
+    const int row = item / n_chunks, chunk = item - row * n_chunks;
+    const int lo = chunk * kChunk;
+    const int n4 = (min(V, lo + kChunk) - lo) >> 2;
+    const bool ok = __all_sync(0xffffffffu, ms::mbar_wait(bars + 8 * s, (k / kStages) & 1, abort_flag,
+                                                          &g_accept_wait_status));
+    Cand best{-INFINITY, INT_MAX};
+    if (ok) {
+      const uint32_t base = sb + s * kStageBytes + lane * 16;
+      auto load4 = [&](int j) -> float4 {
+        float4 x;
+        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];"
+                     : "=f"(x.x), "=f"(x.y), "=f"(x.z), "=f"(x.w)
+                     : "r"(base + static_cast<uint32_t>(j - lane) * 16));
+        return x;
+      };
+      if (lane < n4) {
+        // Branch-free main pass: four running maxima (one per float4 component, each visiting its
+        // indices in increasing order, so "strictly greater" keeps the lowest index of equal
+        // values), started from the lane's first group.  A NaN anywhere shows up in `mix`.
+        float4 x = load4(lane);
+        float bv0 = x.x, bv1 = x.y, bv2 = x.z, bv3 = x.w;
+        int bi0 = lo + 4 * lane, bi1 = bi0 + 1, bi2 = bi0 + 2, bi3 = bi0 + 3;
+        float mix = (x.x + x.y) + (x.z + x.w);
+        bool odd = (mix != mix);
+#pragma unroll 4
+        for (int j = lane + 32; j < n4; j += 32) {
+          x = load4(j);
+          const int i0 = lo + 4 * j;
+          const bool g0 = x.x > bv0, g1 = x.y > bv1, g2 = x.z > bv2, g3 = x.w > bv3;
+          bv0 = g0 ? x.x : bv0;
+          bi0 = g0 ? i0 : bi0;
+          bv1 = g1 ? x.y : bv1;
+          bi1 = g1 ? i0 + 1 : bi1;
+          bv2 = g2 ? x.z : bv2;
+          bi2 = g2 ? i0 + 2 : bi2;
+          bv3 = g3 ? x.w : bv3;
+          bi3 = g3 ? i0 + 3 : bi3;
+          mix = (x.x + x.y) + (x.z + x.w);
+          odd |= (mix != mix);
+        }
+        if (!odd) {
+          best.v = bv0;
+          best.i = bi0;
+          fold(best, bv1, bi1);
+          fold(best, bv2, bi2);
+          fold(best, bv3, bi3);
+        } else {
+          // a NaN (or +inf next to -inf) among this lane's values: the full ordering rule, element by element
+          for (int j = lane; j < n4; j += 32) {
+            x = load4(j);
+            const int i0 = lo + 4 * j;
+            fold(best, x.x, i0);
+            fold(best, x.y, i0 + 1);
+            fold(best, x.z, i0 + 2);
+            fold(best, x.w, i0 + 3);
+          }
+        }
+      }
+      __syncwarp();                              // every lane has read the stage
+      if (lane == 0) ms::mbar_arrive(bars + 8 * (kStages + s));
+      best = warp_best(best);
+    } else {
+      best.i = -1;
+    }
+    if (lane == 0) part[item] = best;
+  }
+}
+
 __global__ void __launch_bounds__(128)
 accept_rows_kernel(const Cand* __restrict__ part, int n_chunks, const int32_t* __restrict__ row_off,
                    int B, const int32_t* __restrict__ draft, int32_t* __restrict__ argmax_out,
@@ -104,9 +239,14 @@ accept_rows_kernel(const Cand* __restrict__ part, int n_chunks, const int32_t* _
   const int r0 = row_off[b], r1 = row_off[b + 1];
   for (int r = r0 + lane; r < r1; r += 32) {
     Cand best{-INFINITY, INT_MAX};
-    for (int c = 0; c < n_chunks; ++c) {
-      const Cand p = part[static_cast<int64_t>(r) * n_chunks + c];
-      fold(best, p.v, p.i);
+    const Cand* __restrict__ pr = part + static_cast<int64_t>(r) * n_chunks;
+    for (int c0 = 0; c0 < n_chunks; c0 += 8) {       // eight loads in flight, then the folds
+      Cand p[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        p[u] = (c0 + u < n_chunks) ? pr[c0 + u] : Cand{-INFINITY, INT_MAX};
+#pragma unroll
+      for (int u = 0; u < 8; ++u) fold(best, p[u].v, p[u].i);
     }
     argmax_out[r] = best.i;
   }
@@ -124,6 +264,33 @@ accept_rows_kernel(const Cand* __restrict__ part, int n_chunks, const int32_t* _
 }
 
 inline int chunks_of(int V) { return (V + kChunk - 1) / kChunk; }
+
+// Pass 1 in whichever form the layout allows.
+int32_t launch_pass1(const float* logits, int64_t ld_v, int vocab, int total_rows, Cand* part, cudaStream_t st) {
+  const int n_chunks = chunks_of(vocab);
+  const int n_items = n_chunks * total_rows;
+  const bool vec = ms::aligned16(logits) && (ld_v % 4 == 0);
+  if (vec && vocab % 4 == 0) {
+    static bool configured[64] = {false};
+    int dev = 0;
+    MS_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev >= 0 && dev < 64 && !configured[dev]) {
+      MS_CUDA_TRY(cudaFuncSetAttribute(argmax_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       kStreamSmem));
+      configured[dev] = true;
+    }
+    const int sms = ms::sm_count();
+    if (sms <= 0) return ms::cuda_status(cudaErrorNoDevice);
+    argmax_stream_kernel<<<n_items < sms ? n_items : sms, kStreamThreads, kStreamSmem, st>>>(
+        logits, ld_v, vocab, n_chunks, n_items, part);
+  } else if (vec) {
+    argmax_chunks_kernel<true><<<static_cast<unsigned>(n_items), kThreads, 0, st>>>(logits, ld_v, vocab, n_chunks, part);
+  } else {
+    argmax_chunks_kernel<false><<<static_cast<unsigned>(n_items), kThreads, 0, st>>>(logits, ld_v, vocab, n_chunks, part);
+  }
+  MS_LAUNCH_CHECK();
+  return MS_OK;
+}
 
 }  // namespace
 
@@ -151,13 +318,8 @@ extern "C" int32_t memosight_accept(const float* logits, int64_t ld_v, int32_t v
   const int n_chunks = chunks_of(vocab);
   Cand* part = static_cast<Cand*>(workspace);
   if (total_rows > 0) {
-    const dim3 grid(static_cast<unsigned>(n_chunks) * static_cast<unsigned>(total_rows));
-    const bool vec = ms::aligned16(logits) && (ld_v % 4 == 0);
-    if (vec)
-      argmax_chunks_kernel<true><<<grid, kThreads, 0, st>>>(logits, ld_v, vocab, n_chunks, part);
-    else
-      argmax_chunks_kernel<false><<<grid, kThreads, 0, st>>>(logits, ld_v, vocab, n_chunks, part);
-    MS_LAUNCH_CHECK();
+    const int32_t rc1 = launch_pass1(logits, ld_v, vocab, total_rows, part, st);
+    if (rc1 != MS_OK) return rc1;
   }
   accept_rows_kernel<<<(batch + 3) / 4, 128, 0, st>>>(part, n_chunks, row_off, batch, draft,
                                                       argmax_out, n_match, n_keep);
@@ -221,13 +383,8 @@ extern "C" int32_t memosight_accept_static(const float* logits, int64_t ld_v, in
   // Nothing in the array has to start at zero: pass 1 writes every (row, chunk) entry that pass 2
   // reads, so whatever an earlier call left behind is overwritten before it is looked at.
   if (total_rows > 0) {
-    const dim3 grid(static_cast<unsigned>(n_chunks) * static_cast<unsigned>(total_rows));
-    const bool vec = ms::aligned16(logits) && (ld_v % 4 == 0);
-    if (vec)
-      argmax_chunks_kernel<true><<<grid, kThreads, 0, st>>>(logits, ld_v, vocab, n_chunks, part);
-    else
-      argmax_chunks_kernel<false><<<grid, kThreads, 0, st>>>(logits, ld_v, vocab, n_chunks, part);
-    MS_LAUNCH_CHECK();
+    const int32_t rc1 = launch_pass1(logits, ld_v, vocab, total_rows, part, st);
+    if (rc1 != MS_OK) return rc1;
   }
   accept_rows_kernel<<<(batch + 3) / 4, 128, 0, st>>>(part, n_chunks, row_off, batch, draft,
                                                       argmax_out, n_match, n_keep);
