@@ -284,7 +284,9 @@ MS_API size_t memosight_accept_workspace_bytes(int32_t total_rows, int32_t vocab
  *              number of candidates that become permanent -- what kv_append takes
  * Row convention: row i of a block holds candidate c_i and predicts the token
  * after it, so draft[i] = c_{i+1}; tokens c_0..c_{n_match} become permanent and
- * argmax_out[row n_match] is the next token. */
+ * argmax_out[row n_match] is the next token.
+ * Every wait inside the kernels is bounded; should one ever run out (a device
+ * fault), the rows concerned get argmax_out = -1, which matches no draft. */
 MS_API int32_t memosight_accept(const float* logits, int64_t ld_v, int32_t vocab, const int32_t* row_off,
                          int32_t batch, int32_t total_rows, const int32_t* draft,
                          int32_t* argmax_out, int32_t* n_match, int32_t* n_keep, void* workspace,
