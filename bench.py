@@ -527,13 +527,14 @@ def run_compress(args, ms, dev, world, rank):
     """Secondary workload: the compression event of long-CoT serving.  Every sequence has just
     finished a 512-token reasoning step; the 170 memory tokens + <o> are forwarded as one causal
     block against the cache (which still holds the verbose step), appended, and the step is
-    evicted.  One "step" = that event for the whole batch, one layer.  Compute-bound: the
+    evicted.  One "step" = that event for the whole batch, one layer; the cache length is put
+    back before every event so that all events are the stated workload.  Compute-bound: the
     roofline is the bf16 tensor peak."""
     assert world == 1, "the compress workload is a single-GPU measurement"
     K, W = args.steps, max(args.warmup, 3)
     B = args.batch if args.batch != 128 else 64
     L0, nq, Hq, Hkv, D = args.kv_len, MEM_TOKENS + 1, 32, 8, 128
-    growth = (K + W) * nq + SEG_LEN + 64
+    growth = nq + SEG_LEN + 64
     cfg = synth.StepConfig("compress", B, Hq, Hkv, D, L0, L0, nq, 0, 5.0e5, 1024, headroom=growth, seed=0x5EED0004)
     inp = synth.make_step_inputs(cfg, device=dev)
     T = B * nq
@@ -558,7 +559,10 @@ def run_compress(args, ms, dev, world, rank):
         a_.record()
         b_.record()
 
+    len0 = inp.kv_len.clone()
+
     def step(ev=None):
+        inp.kv_len.copy_(len0)                       # every event starts from the same cache of L0 entries;
         seg_start.copy_(inp.kv_len)                  # the finished step starts where the cache ended ...
         inp.kv_len.add_(SEG_LEN)                     # ... and its 512 entries are in the cache
         ms.memosight_rope_qk(q_work, ks_work, pos, T, Hq, Hkv, D, cfg.rope_base)
@@ -589,9 +593,9 @@ def run_compress(args, ms, dev, world, rank):
     clocks = sampler.finish()
     elapsed_ms = e0.elapsed_time(e1)
     assert ms.memosight_attn_status(ws) == ms.MS_OK
-    assert inp.kv_len.cpu().tolist() == [L0 + (K + W) * nq] * B
+    assert inp.kv_len.cpu().tolist() == [L0 + nq] * B
     attn_ms = float(np.mean([a_.elapsed_time(b_) for a_, b_ in evs]))
-    l_mid = L0 + SEG_LEN + (W + (K - 1) / 2.0) * nq
+    l_mid = L0 + SEG_LEN
     flops = 4.0 * B * Hq * D * nq * (l_mid + (nq + 1) / 2.0)       # visible keys: cache + causal half
     sustained, burst, kind = peak_tensor()
     achieved = flops / (attn_ms * 1e-3) / 1e12
@@ -601,7 +605,7 @@ def run_compress(args, ms, dev, world, rank):
         "steps": K, "warmup": W, "ms_per_step": elapsed_ms / K, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": f"compression event, 8B-shape layer H_q={Hq} H_kv={Hkv} D={D}, batch {B}, cache "
-                               f"{L0} + a {SEG_LEN}-token step, block of {nq} causal tokens, 1 layer",
+                               f"{L0} + a {SEG_LEN}-token step (the same at every event), block of {nq} causal tokens, 1 layer",
                    "global_batch": B, "kv_len": L0, "block": nq,
                    "l2": "K/V of one sequence-layer (69 MB) is re-read by the 6 row tiles of a KV head, mostly "
                          "from L2; no flush"},
