@@ -261,6 +261,38 @@ def test_accept_unplanted_ties_nan_inf_and_unaligned_rows():
     _accept_both(b.logits, cfg.vocab, a.row_off.tolist(), a.draft.tolist())
 
 
+@pytest.mark.parametrize("V", [4, 132, 8192, 8204, 3 * 8192 + 512, 151936])
+def test_accept_streaming_form_ordering_rule(V):
+    """16-byte-aligned rows and a vocabulary that is a multiple of 4 take the streaming pass 1
+    (bulk copies into a shared-memory ring, branch-free per-lane maxima): ties across lanes, chunks
+    and float4 components, NaN, +-inf and all-equal rows must come out by the same ordering rule."""
+    cfg = synth.StepConfig("acc3", 12, 4, 2, 64, 8, 8, 3, 2, 1e4, V, seed=7)
+    a = synth.make_accept_inputs(cfg, plant=False)
+    assert a.ld_v % 4 == 0
+    lg = a.logits
+    T = lg.shape[0]
+    assert T >= 14
+    col = lambda x: min(max(int(x), 0), V - 1)
+    lg[1, [col(9), col(V - 3)]] = 50.0                      # same maximum early and in the last chunk: first wins
+    lg[2, [col(V - 1), col(0)]] = 50.0
+    lg[3, [col(128 + 1), col(128 + 2), col(4 * 32 * 5 + 3)]] = 60.0   # same lane, neighbouring components, later group
+    lg[4, :] = float("-inf")                                # nothing beats -inf: index 0
+    lg[5, col(77)] = float("inf")
+    lg[6, [col(30), col(V - 2)]] = float("nan")             # first NaN wins, also over +inf
+    lg[6, col(10)] = float("inf")
+    lg[7, :] = 0.0
+    lg[7, col(5)] = -0.0                                    # -0 == +0: index 0
+    lg[8, col(V // 2)] = float("inf")
+    lg[8, col(V // 2 + 1)] = float("-inf")                  # +inf and -inf in one float4 group: not a NaN
+    lg[9, :] = -3.0e38
+    lg[9, col(V - 1)] = -2.9e38
+    lg[10, col(3)] = float("nan")
+    lg[11, [col(8191), col(8192)]] = 70.0                   # across a chunk boundary
+    lg[12, col(V - 1)] = float("nan")
+    lg[13, :] = float("nan")
+    _accept_both(lg, V, a.row_off.tolist(), a.draft.tolist())
+
+
 def test_accept_llama_vocab_config():
     cfg = synth.LLAMA8B_RAGGED
     a = synth.make_accept_inputs(cfg, device=DEV)
