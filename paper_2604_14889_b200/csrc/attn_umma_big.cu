@@ -440,7 +440,8 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
         }
       }
       if (!wait_all(bars + 8 * (kBbSFull + pb), (it >> 1) & 1)) { ok = false; break; }
-      if (it >= 2 && !wait_all(bars + 8 * (kBbPvDone + pb), ((it >> 1) - 1) & 1)) { ok = false; break; }
+      // P buffer `pb` is free as well: the commit that completed S(it) tracks every tcgen05 operation
+      // the issuing thread started before it, and O += P V of tile it - 2 is one of them
       tc_fence_after();
       const int nv = w.nvalid;
       const bool is_step = w.step_idx >= 0;
