@@ -208,6 +208,13 @@ __device__ __forceinline__ float max_cols(const float (&v)[kBCw]) {
   return fmaxf(fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3])), fmaxf(fmaxf(m[4], m[5]), fmaxf(m[6], m[7])));
 }
 
+// mbarrier.arrive under a predicate, without a branch.
+__device__ __forceinline__ void mbar_arrive_if(bool pred, uint32_t bar) {
+  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %1, 0;\n\t@p mbarrier.arrive.shared::cta.b64 _, [%0];\n\t}"
+               ::"r"(bar), "r"(static_cast<uint32_t>(pred))
+               : "memory");
+}
+
 // ---------------------------------------------------------------- kernel
 
 __global__ void __launch_bounds__(kBThreads, 1)
@@ -411,7 +418,7 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
     // bounded barrier of all softmax warps (also publishes their shared-memory writes)
     auto sync_all = [&]() -> bool {
       __syncwarp();
-      if (lane == 0) mbar_arrive(bars + 8 * kBbAll);
+      mbar_arrive_if(lane == 0, bars + 8 * kBbAll);
       const bool good = wait_all(bars + 8 * kBbAll, all_phase & 1);
       ++all_phase;
       return good;
@@ -530,7 +537,7 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
       fence_async_smem();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bars + 8 * (kBbPFull + pb));
+      mbar_arrive_if(lane == 0, bars + 8 * (kBbPFull + pb));
 
       if (w.last) {
         // ---- end of the item: the unit, or this chunk of it ----
