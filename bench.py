@@ -227,13 +227,18 @@ def oracle_step_sample(cfg, n_seqs, seed_shift=0, gen_device="cpu"):
     return step, oracle.threads()
 
 
-def cpu_baseline(cfg, n_seqs, gen_device):
+def cpu_baseline(cfg, n_seqs, gen_device, min_seconds=10.0, max_steps=8):
+    """The oracle as it stands on the host cores: whole steps of a sample of the batch, repeated
+    until about ten seconds of CPU work have been timed."""
     step, cores = oracle_step_sample(cfg, n_seqs, gen_device=gen_device)
+    tokens, n_steps = 0, 0
     t0 = time.perf_counter()
-    tokens = step()
+    while n_steps < max_steps and (n_steps == 0 or time.perf_counter() - t0 < min_seconds):
+        tokens += step()
+        n_steps += 1
     dt = time.perf_counter() - t0
     return {"value": tokens / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": f"one whole step (rope, attention, accept, append, compaction) of {n_seqs} of the "
+            "sample": f"{n_steps} whole steps (rope, attention, accept, append, compaction) of {n_seqs} of the "
                       f"{cfg.batch} sequences (L={cfg.len_lo}, {cfg.n_q} block rows each), {dt:.1f} s"}
 
 
