@@ -680,7 +680,8 @@ def run_e2e(ms, n_e2e, first, cfg, inp, acc, sched, seg_start, seg_len, ws, wsb,
     d2h = h_out.numel() * 2 + h_am.numel() * 4 + h_nm.numel() * 4
     return {"value": T * n_e2e / dt, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
             "steps": n_e2e, "ms_per_step": dt / n_e2e * 1e3,
-            "call": "memosight_step_host (pinned host buffers, one stream, host sync after every step)"}
+            "call": "memosight_step_host (pinned host buffers; the logits copy runs on the library's copy stream beside the "
+                    "attention; host sync after every step)"}
 
 
 if __name__ == "__main__":

@@ -399,6 +399,11 @@ MS_API int32_t memosight_decode_commit_compress(const memosight_decode_state* st
  * asynchronous), runs RoPE -> step attention -> greedy accept -> append of the
  * accepted candidates (-> optional compaction) on `stream`, and copies the results
  * back.  All device pointers are caller-owned staging buffers of the stated sizes.
+ * The logits are copied on a stream of the library's own (created, with two
+ * events, at the first call on a device) beside RoPE and the attention, and joined
+ * into `stream` before the accept; calls for one device share that stream and the
+ * events, so issue them one after the other, not from several threads at once,
+ * and make the first call on a device outside any stream capture.
  * The call returns after queueing; synchronise `stream` before reading h_*. */
 typedef struct memosight_step_host_params {
   uint32_t struct_size;          /* sizeof(memosight_step_host_params)                         */

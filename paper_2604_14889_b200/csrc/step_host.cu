@@ -1,8 +1,45 @@
 // One whole decode step driven from host-resident step data: copies in, the
 // kernels of the hot path in their order (Algorithm 1: forward pass attention,
 // greedy accept, S <- S (+) A, optional UpdateCache), copies out.  Pure
-// sequencing of the other entry points on one stream.
+// sequencing of the other entry points on the caller's stream -- except that the
+// logits, by far the largest input and needed only by the accept, are copied on a
+// second stream of the library's own while RoPE and the attention run, and joined
+// back by an event before the accept.
+#include <mutex>
+
 #include "common.cuh"
+
+namespace {
+
+struct CopyLane {
+  cudaStream_t stream = nullptr;
+  cudaEvent_t fork = nullptr, join = nullptr;
+};
+
+// One copy stream and two events per device, created at the first call on that device.
+int32_t copy_lane(CopyLane** out) {
+  static std::mutex mu;
+  static CopyLane lanes[64];
+  int dev = 0;
+  MS_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return MS_ERR_UNSUPPORTED_SHAPE;
+  std::lock_guard<std::mutex> lock(mu);
+  CopyLane& l = lanes[dev];
+  if (!l.stream) {
+    cudaStream_t s = nullptr;
+    cudaEvent_t f = nullptr, j = nullptr;
+    MS_CUDA_TRY(cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking));
+    MS_CUDA_TRY(cudaEventCreateWithFlags(&f, cudaEventDisableTiming));
+    MS_CUDA_TRY(cudaEventCreateWithFlags(&j, cudaEventDisableTiming));
+    l.fork = f;
+    l.join = j;
+    l.stream = s;
+  }
+  *out = &l;
+  return MS_OK;
+}
+
+}  // namespace
 
 extern "C" int32_t memosight_step_host(const memosight_step_host_params* p,
                                        memosight_stream_t stream) {
@@ -27,10 +64,18 @@ extern "C" int32_t memosight_step_host(const memosight_step_host_params* p,
   MS_CUDA_TRY(cudaMemcpyAsync(const_cast<void*>(a.k_step), p->h_k_step, kv_bytes, cudaMemcpyHostToDevice, st));
   MS_CUDA_TRY(cudaMemcpyAsync(const_cast<void*>(a.v_step), p->h_v_step, kv_bytes, cudaMemcpyHostToDevice, st));
   MS_CUDA_TRY(cudaMemcpyAsync(p->d_pos_id, p->h_pos_id, sizeof(int32_t) * T, cudaMemcpyHostToDevice, st));
+  CopyLane* lane = nullptr;
   if (p->vocab > 0) {
+    // the logits go their own way: behind whatever `stream` holds now (the previous step's accept
+    // may still read the staging buffer), beside RoPE and the attention, back in before the accept
+    const int32_t rc_lane = copy_lane(&lane);
+    if (rc_lane != MS_OK) return rc_lane;
+    MS_CUDA_TRY(cudaEventRecord(lane->fork, st));
+    MS_CUDA_TRY(cudaStreamWaitEvent(lane->stream, lane->fork, 0));
     MS_CUDA_TRY(cudaMemcpyAsync(p->d_logits, p->h_logits, sizeof(float) * static_cast<size_t>(T) * p->ld_v,
-                                cudaMemcpyHostToDevice, st));
-    MS_CUDA_TRY(cudaMemcpyAsync(p->d_draft, p->h_draft, sizeof(int32_t) * T, cudaMemcpyHostToDevice, st));
+                                cudaMemcpyHostToDevice, lane->stream));
+    MS_CUDA_TRY(cudaMemcpyAsync(p->d_draft, p->h_draft, sizeof(int32_t) * T, cudaMemcpyHostToDevice, lane->stream));
+    MS_CUDA_TRY(cudaEventRecord(lane->join, lane->stream));
   }
   // ---- the hot path
   int32_t rc = memosight_rope_qk(const_cast<void*>(a.q), const_cast<void*>(a.k_step), p->d_pos_id, T,
@@ -40,6 +85,7 @@ extern "C" int32_t memosight_step_host(const memosight_step_host_params* p,
   rc = memosight_attn_step(&a, stream);
   if (rc != MS_OK) return rc;
   if (p->vocab > 0) {
+    MS_CUDA_TRY(cudaStreamWaitEvent(st, lane->join, 0));
     rc = memosight_accept(p->d_logits, p->ld_v, p->vocab, a.q_off, B, T, p->d_draft, p->d_argmax,
                           p->d_n_match, p->d_n_keep, p->accept_workspace, p->accept_workspace_bytes,
                           stream);
