@@ -429,7 +429,118 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
       for (int g = 1; g < kBWg; ++g) m = fmaxf(m, arr[g * kTile + r]);
       return m;
     };
+    // One tile from the scores in tensor memory to P handed over (S(it) is complete; the P buffer is
+    // free with it: the commit behind S(it) tracks every earlier tcgen05 operation of the issuing
+    // thread, O += P V of tile it - 2 among them).  `masked`: ragged or step-local tile.
+    auto tile_body = [&](const bool masked, const bool opens_item, const int nv, const bool is_step,
+                         const int step_idx, const int it) -> bool {
+      const int pb = it & 1;
+      tc_fence_after();
+      if (masked && (nv & 15)) {
+        // V rows past the valid keys hold foreign or stale bytes; P is 0 there but 0 * NaN is NaN
+        const int use = 2 * it + 1, buf = use % kBKv;
+        if (!wait_all(bars + 8 * (kBbKvFull + buf), (use / kBKv) & 1)) return false;
+        const uint32_t va = sb + kBOffKv + buf * kBKvBytes;
+        const int n_rows = ((nv + 15) & ~15) - nv;
+        for (int x = wg * kTile + r; x < n_rows * HALVES * 8; x += kBWg * kTile) {
+          const int rr = nv + x / (HALVES * 8), cc = x % (HALVES * 8);
+          const uint32_t addr = va + (cc >> 3) * kBHalf + rr * 128 + ((cc & 7) << 4);
+          asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(addr), "r"(0u) : "memory");
+        }
+      }
+      // this warpgroup's score columns of the row; invisible keys become -inf
+      const uint32_t s_addr = lane_addr + kBColS + pb * kTile + wg * kBCw;
+      const int key0 = (is_step ? step_idx * kTile : 0) + wg * kBCw;   // step-local index of column 0
+      float v[kBCw];
+      if (masked)
+        big_load_scores<true>(s_addr, v, wg * kBCw, nv, is_step, tok, key0, w.s.n_c, anc,
+                              a.tok_kind ? a.tok_kind + w.s.r0 : nullptr, a.tok_kind ? a.tok_step + w.s.r0 : nullptr);
+      else
+        big_load_scores<false>(s_addr, v, 0, kTile, false, 0, 0, 0, 0);
+      if (opens_item) {
+        // new unit: reference = exact maximum of the first tile over all column groups
+        s_mx[wg * kTile + r] = max_cols(v);
+        if (!sync_all()) return false;
+        const float m = max_of_groups(s_mx);
+        m_ref = (m == -INFINITY) ? 0.f : m * a.scale_log2;
+        l_part = 0.f;
+      }
+      // p = 2^(s*scale - m_ref) as bf16 into this row of the P tile; the row's partial sum over
+      // this group's keys
+      const uint32_t p_row = sb + kBOffP + pb * kBPBytes + ((wg * kBCw) >> 6) * kBHalf + r * 128;
+      const int chunk0 = ((wg * kBCw) & 63) >> 3;             // first 16-byte chunk inside the 64-key half
+      auto p_pass = [&]() -> float {
+        float ls[4] = {0.f, 0.f, 0.f, 0.f};
+  #pragma unroll
+        for (int c = 0; c < kBCw / 8; ++c) {
+          float p[8];
+  #pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            p[e] = ex2(fmaf(v[c * 8 + e], a.scale_log2, -m_ref));
+            ls[e & 3] += p[e];
+          }
+          const uint32_t addr = p_row + (((chunk0 + c) ^ rx) << 4);
+          asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(pack2(p[0], p[1])),
+                       "r"(pack2(p[2], p[3])), "r"(pack2(p[4], p[5])), "r"(pack2(p[6], p[7]))
+                       : "memory");
+        }
+        return (ls[0] + ls[1]) + (ls[2] + ls[3]);
+      };
+      float tsum = p_pass();
+      // A score that outgrew the row reference by ~2^48 shows in the sum (so do inf and NaN); the
+      // softmax warps agree on it before anyone hands P over
+      if (!opens_item && __any_sync(0xffffffffu, row_ok && !(tsum < kBGrowSum)) && lane == 0)
+        *grow_flag = it + 1;
+      if (!sync_all()) return false;
+      if (*grow_flag == it + 1) {
+        // ---- rare: move the row references up; rescale O (this group's columns) and the sums ----
+        s_mx[wg * kTile + r] = max_cols(v);
+        if (!sync_all()) return false;
+        const float m = max_of_groups(s_mx);
+        const float m_new = (m == -INFINITY) ? m_ref : fmaxf(m_ref, m * a.scale_log2);
+        const float alpha = ex2(m_ref - m_new);
+        m_ref = m_new;
+        l_part *= alpha;
+        if (!wait_all(bars + 8 * (kBbPvDone + ((it - 1) & 1)), ((it - 1) >> 1) & 1)) return false;
+        tc_fence_after();
+  #pragma unroll 1
+        for (int c = 0; c < kBCw / 32; ++c) {
+          uint32_t o[32];
+          tmem_ld32(lane_addr + kBColO + wg * kBCw + c * 32, o);
+          tmem_ld_wait(o);
+  #pragma unroll
+          for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+          tmem_st32(lane_addr + kBColO + wg * kBCw + c * 32, o);
+        }
+        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+        tsum = p_pass();
+        if (!sync_all()) return false;     // s_mx may be rewritten from here on
+      }
+      l_part += tsum;
+      fence_async_smem();
+      tc_fence_before();
+      __syncwarp();
+      mbar_arrive_if(lane == 0, bars + 8 * (kBbPFull + pb));
+      return true;
+    };
     while (ok && w.it < n_iter) {
+      // ---- a run of plain tiles -- full cache tiles that neither open nor close the item -- needs
+      //      none of the walker: most tiles of a long cache go through this loop
+      if (w.ti > w.ti_lo) {
+        const int stop = min(w.s.L / kTile, w.ti_hi - 1);
+        while (w.ti < stop) {
+          const int it = w.it;
+          if (!wait_all(bars + 8 * (kBbSFull + (it & 1)), (it >> 1) & 1) ||
+              !tile_body(false, false, kTile, false, 0, it)) {
+            ok = false;
+            break;
+          }
+          ++w.ti;
+          ++w.it;
+          ++w.piece_j;
+        }
+        if (!ok) break;
+      }
       bwalk_tile(w);
       const int it = w.it, pb = it & 1;
       if (w.first) {
@@ -447,97 +558,11 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
         }
       }
       if (!wait_all(bars + 8 * (kBbSFull + pb), (it >> 1) & 1)) { ok = false; break; }
-      // P buffer `pb` is free as well: the commit that completed S(it) tracks every tcgen05 operation
-      // the issuing thread started before it, and O += P V of tile it - 2 is one of them
-      tc_fence_after();
-      const int nv = w.nvalid;
-      const bool is_step = w.step_idx >= 0;
-      const bool masked = is_step || nv < kTile;
-      if (masked && (nv & 15)) {
-        // V rows past the valid keys hold foreign or stale bytes; P is 0 there but 0 * NaN is NaN
-        const int use = 2 * it + 1, buf = use % kBKv;
-        if (!wait_all(bars + 8 * (kBbKvFull + buf), (use / kBKv) & 1)) { ok = false; break; }
-        const uint32_t va = sb + kBOffKv + buf * kBKvBytes;
-        const int n_rows = ((nv + 15) & ~15) - nv;
-        for (int x = wg * kTile + r; x < n_rows * HALVES * 8; x += kBWg * kTile) {
-          const int rr = nv + x / (HALVES * 8), cc = x % (HALVES * 8);
-          const uint32_t addr = va + (cc >> 3) * kBHalf + rr * 128 + ((cc & 7) << 4);
-          asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(addr), "r"(0u) : "memory");
-        }
+      {
+        const int nv = w.nvalid;
+        const bool is_step = w.step_idx >= 0;
+        if (!tile_body(is_step || nv < kTile, w.piece_j == 0, nv, is_step, w.step_idx, it)) { ok = false; break; }
       }
-      // this warpgroup's score columns of the row; invisible keys become -inf
-      const uint32_t s_addr = lane_addr + kBColS + pb * kTile + wg * kBCw;
-      const int key0 = (is_step ? w.step_idx * kTile : 0) + wg * kBCw;   // step-local index of column 0
-      float v[kBCw];
-      if (masked)
-        big_load_scores<true>(s_addr, v, wg * kBCw, nv, is_step, tok, key0, w.s.n_c, anc,
-                              a.tok_kind ? a.tok_kind + w.s.r0 : nullptr, a.tok_kind ? a.tok_step + w.s.r0 : nullptr);
-      else
-        big_load_scores<false>(s_addr, v, 0, kTile, false, 0, 0, 0, 0);
-      if (w.piece_j == 0) {
-        // new unit: reference = exact maximum of the first tile over all column groups
-        s_mx[wg * kTile + r] = max_cols(v);
-        if (!sync_all()) { ok = false; break; }
-        const float m = max_of_groups(s_mx);
-        m_ref = (m == -INFINITY) ? 0.f : m * a.scale_log2;
-        l_part = 0.f;
-      }
-      // p = 2^(s*scale - m_ref) as bf16 into this row of the P tile; the row's partial sum over
-      // this group's keys
-      const uint32_t p_row = sb + kBOffP + pb * kBPBytes + ((wg * kBCw) >> 6) * kBHalf + r * 128;
-      const int chunk0 = ((wg * kBCw) & 63) >> 3;             // first 16-byte chunk inside the 64-key half
-      auto p_pass = [&]() -> float {
-        float ls[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-        for (int c = 0; c < kBCw / 8; ++c) {
-          float p[8];
-#pragma unroll
-          for (int e = 0; e < 8; ++e) {
-            p[e] = ex2(fmaf(v[c * 8 + e], a.scale_log2, -m_ref));
-            ls[e & 3] += p[e];
-          }
-          const uint32_t addr = p_row + (((chunk0 + c) ^ rx) << 4);
-          asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(pack2(p[0], p[1])),
-                       "r"(pack2(p[2], p[3])), "r"(pack2(p[4], p[5])), "r"(pack2(p[6], p[7]))
-                       : "memory");
-        }
-        return (ls[0] + ls[1]) + (ls[2] + ls[3]);
-      };
-      float tsum = p_pass();
-      // A score that outgrew the row reference by ~2^48 shows in the sum (so do inf and NaN); the
-      // softmax warps agree on it before anyone hands P over
-      if (w.piece_j > 0 && __any_sync(0xffffffffu, row_ok && !(tsum < kBGrowSum)) && lane == 0)
-        *grow_flag = it + 1;
-      if (!sync_all()) { ok = false; break; }
-      if (*grow_flag == it + 1) {
-        // ---- rare: move the row references up; rescale O (this group's columns) and the sums ----
-        s_mx[wg * kTile + r] = max_cols(v);
-        if (!sync_all()) { ok = false; break; }
-        const float m = max_of_groups(s_mx);
-        const float m_new = (m == -INFINITY) ? m_ref : fmaxf(m_ref, m * a.scale_log2);
-        const float alpha = ex2(m_ref - m_new);
-        m_ref = m_new;
-        l_part *= alpha;
-        if (!wait_all(bars + 8 * (kBbPvDone + ((it - 1) & 1)), ((it - 1) >> 1) & 1)) { ok = false; break; }
-        tc_fence_after();
-#pragma unroll 1
-        for (int c = 0; c < kBCw / 32; ++c) {
-          uint32_t o[32];
-          tmem_ld32(lane_addr + kBColO + wg * kBCw + c * 32, o);
-          tmem_ld_wait(o);
-#pragma unroll
-          for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-          tmem_st32(lane_addr + kBColO + wg * kBCw + c * 32, o);
-        }
-        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-        tsum = p_pass();
-        if (!sync_all()) { ok = false; break; }     // s_mx may be rewritten from here on
-      }
-      l_part += tsum;
-      fence_async_smem();
-      tc_fence_before();
-      __syncwarp();
-      mbar_arrive_if(lane == 0, bars + 8 * (kBbPFull + pb));
 
       if (w.last) {
         // ---- end of the item: the unit, or this chunk of it ----
