@@ -365,6 +365,55 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
     };
     ok = issue_qk();
     while (ok && wp.it < n_iter) {
+      // ---- a run of plain tiles needs neither walker: S of a tile that is neither the first nor the
+      //      last of its item, O += P V of a full cache tile that is not the first
+      if (wq.item == wp.item && wp.ti > wp.ti_lo && wq.it == wp.it + 1) {
+        int n_run = min(wq.ti_hi - 1 - wq.ti, wp.s.L / kTile - wp.ti);
+        int it = wp.it;
+        for (; n_run > 0; --n_run, ++it) {
+          // S(it + 1)
+          if (!mbar_wait(bars + 8 * (kBbKvFull + rk.buf), rk.par, abort_flag, status)) { ok = false; break; }
+          tc_fence_after();
+          {
+            const uint32_t k_lo = k_lo0 + rk.buf * (kBKvBytes >> 4);
+            const uint32_t d_s = tmem + kBColS + ((it + 1) & 1) * kTile;
+#pragma unroll
+            for (int ks = 0; ks < KSTEPS; ++ks) {
+              const uint32_t off = (ks >> 2) * (kBHalf >> 4) + (ks & 3) * 2;
+              umma_bf16_lo(d_s, q_lo + off, k_lo + off, idesc_qk, ks > 0);
+            }
+            umma_commit(bars + 8 * (kBbKvEmpty + rk.buf));
+            umma_commit(bars + 8 * (kBbSFull + ((it + 1) & 1)));
+            rk.step(2);
+          }
+          // O += P V (it)
+          if (!mbar_wait(bars + 8 * (kBbPFull + (it & 1)), (it >> 1) & 1, abort_flag, status) ||
+              !mbar_wait(bars + 8 * (kBbKvFull + rv.buf), rv.par, abort_flag, status)) {
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          {
+            const uint32_t p_lo = p_lo0 + (it & 1) * (kBPBytes >> 4);
+            const uint32_t v_lo = v_lo0 + rv.buf * (kBKvBytes >> 4);
+#pragma unroll
+            for (int j = 0; j < kTile / 16; ++j)
+              umma_bf16_lo(tmem + kBColO, p_lo + (j >> 2) * (kBHalf >> 4) + (j & 3) * 2, v_lo + j * (2048 >> 4),
+                           idesc_pv, 1u);
+            umma_commit(bars + 8 * (kBbKvEmpty + rv.buf));
+            umma_commit(bars + 8 * (kBbPvDone + (it & 1)));
+            rv.step(2);
+          }
+        }
+        if (!ok) break;
+        const int done = it - wp.it;
+        wq.ti += done;
+        wq.it += done;
+        wq.piece_j += done;
+        wp.ti += done;
+        wp.it += done;
+        wp.piece_j += done;
+      }
       if (wq.it < n_iter && !issue_qk()) { ok = false; break; }
       bwalk_tile(wp);
       const int it = wp.it;
