@@ -292,6 +292,34 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
     RingPos rp;
     rp.init(0, kBKv);
     while (w.it < n_iter) {
+      // ---- a run of cache tiles behind the item's first tile: K and V of tile after tile, no walker
+      if (w.ti > w.ti_lo) {
+        const int stop = min(w.s.cache_tiles, w.ti_hi);
+        const int n_run = stop - w.ti;
+        int y = static_cast<int>(w.s.slot_off) + w.ti * kTile;
+        for (int k = 0; k < 2 * n_run; ++k) {
+          const int buf = rp.buf;
+          if (!mbar_wait(bars + 8 * (kBbKvEmpty + buf), rp.par ^ 1u, abort_flag, status)) { ok = false; break; }
+          rp.step(1);
+          fence_async_smem();
+          const uint32_t dst = sb + kBOffKv + buf * kBKvBytes;
+          const uint32_t bar = bars + 8 * (kBbKvFull + buf);
+          mbar_arrive_expect_tx(bar, static_cast<uint32_t>(kBKvBytes));
+          const CUtensorMap* map = (k & 1) ? &map_v : &map_k;
+          tma_load_3d(dst, map, bar, 0, y, w.h);
+          tma_load_3d(dst + kBHalf, map, bar, 64, y, w.h);
+          ++uses;
+          y += (k & 1) * kTile;
+        }
+        if (!ok) break;
+        if (n_run > 0) {
+          w.ti += n_run - 1;            // bwalk_next moves past the run's last tile (and on to the next item)
+          w.it += n_run - 1;
+          w.piece_j += n_run - 1;
+          bwalk_next(a, w, pre);
+          continue;
+        }
+      }
       bwalk_tile(w);
       if (w.first) {
         // one Q buffer: every Q K^T of the previous unit must have read it
