@@ -45,8 +45,8 @@ constexpr int kBSmem = kBOffMisc + kBMiscBytes;
 static_assert(kBSmem <= 227 * 1024, "shared memory budget");
 
 enum : int {
-  kBbKvFull = 0, kBbKvEmpty = kBKv, kBbQFull = 2 * kBKv, kBbQEmpty, kBbSFull, kBbPFull = kBbSFull + 2,
-  kBbPvDone = kBbPFull + 2, kBbAll = kBbPvDone + 2, kBbDrain, kBbCount
+  kBbKvFull = 0, kBbKvEmpty = kBKv, kBbQFull = 2 * kBKv, kBbQEmpty, kBbPFull, kBbAll = kBbPFull + 2, kBbDrain,
+  kBbCount
 };
 static_assert(kBbCount * 8 <= kBMiscScalars, "barriers overflow their slot");
 
@@ -262,9 +262,7 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
     mbar_init(bars + 8 * kBbQFull, 1);
     mbar_init(bars + 8 * kBbQEmpty, 1);
     for (int i = 0; i < 2; ++i) {
-      mbar_init(bars + 8 * (kBbSFull + i), 1);
       mbar_init(bars + 8 * (kBbPFull + i), 4 * kBWg);
-      mbar_init(bars + 8 * (kBbPvDone + i), 1);
     }
     mbar_init(bars + 8 * kBbAll, 4 * kBWg);
     mbar_init(bars + 8 * kBbDrain, 1);
@@ -385,7 +383,6 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
         umma_bf16_lo(d_s, q_lo + off, k_lo + off, idesc_qk, ks > 0);
       }
       umma_commit(bars + 8 * (kBbKvEmpty + rk.buf));
-      umma_commit(bars + 8 * (kBbSFull + (it & 1)));
       if (wq.last) umma_commit(bars + 8 * kBbQEmpty);
       rk.step(2);
       bwalk_next(a, wq, pre);
@@ -411,7 +408,6 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
               umma_bf16_lo(d_s, q_lo + off, k_lo + off, idesc_qk, ks > 0);
             }
             umma_commit(bars + 8 * (kBbKvEmpty + rk.buf));
-            umma_commit(bars + 8 * (kBbSFull + ((it + 1) & 1)));
             rk.step(2);
           }
           // O += P V (it)
@@ -429,7 +425,6 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
               umma_bf16_lo(tmem + kBColO, p_lo + (j >> 2) * (kBHalf >> 4) + (j & 3) * 2, v_lo + j * (2048 >> 4),
                            idesc_pv, 1u);
             umma_commit(bars + 8 * (kBbKvEmpty + rv.buf));
-            umma_commit(bars + 8 * (kBbPvDone + (it & 1)));
             rv.step(2);
           }
         }
@@ -467,7 +462,6 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
                        idesc_pv, j == 0 ? acc0 : 1u);
       }
       umma_commit(bars + 8 * (kBbKvEmpty + rv.buf));
-      umma_commit(bars + 8 * (kBbPvDone + (it & 1)));
       rv.step(2);
       bwalk_next(a, wp, pre);
     }
@@ -489,6 +483,14 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
     bool row_ok = false;
     uint32_t all_phase = 0;
     bool ok = true;
+    // "S(it) is complete" and "O += P V of tile it is complete" need no barriers of their own: the
+    // commits that release the tile's K buffer (ring use 2 it) and V buffer (use 2 it + 1) are those
+    // events, and with four ring buffers the phase parity is (it >> 1) & 1 for both.  A waiter is
+    // never two phases behind: the buffer's next use belongs to tile it + 2, whose S needs this
+    // tile's P handed over and whose PV needs its own.
+    static_assert(kBKv == 4, "the ring position of a tile's K and V buffers is taken from its parity");
+    auto bar_s_full = [&](int it) -> uint32_t { return bars + 8 * (kBbKvEmpty + 2 * (it & 1)); };
+    auto bar_pv_done = [&](int it) -> uint32_t { return bars + 8 * (kBbKvEmpty + 2 * (it & 1) + 1); };
     auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {
       return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, status));
     };
@@ -578,7 +580,7 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
         const float alpha = ex2(m_ref - m_new);
         m_ref = m_new;
         l_part *= alpha;
-        if (!wait_all(bars + 8 * (kBbPvDone + ((it - 1) & 1)), ((it - 1) >> 1) & 1)) return false;
+        if (!wait_all(bar_pv_done(it - 1), ((it - 1) >> 1) & 1)) return false;
         tc_fence_after();
   #pragma unroll 1
         for (int c = 0; c < kBCw / 32; ++c) {
@@ -607,7 +609,7 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
         const int stop = min(w.s.L / kTile, w.ti_hi - 1);
         while (w.ti < stop) {
           const int it = w.it;
-          if (!wait_all(bars + 8 * (kBbSFull + (it & 1)), (it >> 1) & 1) ||
+          if (!wait_all(bar_s_full(it), (it >> 1) & 1) ||
               !tile_body(false, false, kTile, false, 0, it)) {
             ok = false;
             break;
@@ -619,7 +621,7 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
         if (!ok) break;
       }
       bwalk_tile(w);
-      const int it = w.it, pb = it & 1;
+      const int it = w.it;
       if (w.first) {
         const int tok0 = w.rt * tpt;
         rows = (min(w.s.n_q, tok0 + tpt) - tok0) * a.G;
@@ -634,7 +636,7 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
           anc = 0;
         }
       }
-      if (!wait_all(bars + 8 * (kBbSFull + pb), (it >> 1) & 1)) { ok = false; break; }
+      if (!wait_all(bar_s_full(it), (it >> 1) & 1)) { ok = false; break; }
       {
         const int nv = w.nvalid;
         const bool is_step = w.step_idx >= 0;
@@ -648,7 +650,7 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
         float l_row = 0.f;
 #pragma unroll
         for (int g = 0; g < kBWg; ++g) l_row += s_lp[g * kTile + r];
-        if (!wait_all(bars + 8 * (kBbPvDone + pb), (it >> 1) & 1)) { ok = false; break; }
+        if (!wait_all(bar_pv_done(it), (it >> 1) & 1)) { ok = false; break; }
         tc_fence_after();
         const int i = tok, g = r % a.G;
         const int64_t orow = static_cast<int64_t>(w.s.r0 + (row_ok ? i : 0)) * a.H_q + w.h * a.G + g;
