@@ -167,6 +167,14 @@ __device__ __forceinline__ void bwalk_next(const AttnArgs& a, BigWalk& w, const 
   if (++w.ti == w.ti_hi) bwalk_advance(a, w, pre);
 }
 
+// Number of leading step-local key tiles of an item that need no mask: every key of such a tile is a
+// candidate that precedes every token of the row tile, and all its rows are candidates (default
+// anchors, no training-time mask) -- the tiles left of the diagonal of a prefill or compression block.
+__device__ __forceinline__ int big_plain_step_tiles(const AttnArgs& a, const BigSeq& s, int rt, int tpt) {
+  const int tok0 = rt * tpt, tok_end = min(s.n_q, tok0 + tpt);
+  return (!a.tok_kind && !a.anchor && tok_end <= s.n_c) ? tok0 / kTile : 0;
+}
+
 __device__ __host__ inline size_t big_slot_floats() { return static_cast<size_t>(kTile) * (kBD + 2); }
 
 // The warpgroup's 64 score columns of one row, from tensor memory into v[]; with kMasked the
@@ -290,33 +298,46 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
     RingPos rp;
     rp.init(0, kBKv);
     while (w.it < n_iter) {
-      // ---- a run of cache tiles behind the item's first tile: K and V of tile after tile, no walker
+      // ---- the item's tiles behind its first: K and V of tile after tile, no walker
       if (w.ti > w.ti_lo) {
-        const int stop = min(w.s.cache_tiles, w.ti_hi);
-        const int n_run = stop - w.ti;
-        int y = static_cast<int>(w.s.slot_off) + w.ti * kTile;
-        for (int k = 0; k < 2 * n_run; ++k) {
+        const int ct = w.s.cache_tiles, n_run = w.ti_hi - w.ti;
+        const int n_cache = max(0, min(ct, w.ti_hi) - w.ti);
+        auto ring_slot = [&](uint32_t& dst, uint32_t& bar) -> bool {
           const int buf = rp.buf;
-          if (!mbar_wait(bars + 8 * (kBbKvEmpty + buf), rp.par ^ 1u, abort_flag, status)) { ok = false; break; }
+          if (!mbar_wait(bars + 8 * (kBbKvEmpty + buf), rp.par ^ 1u, abort_flag, status)) return false;
           rp.step(1);
           fence_async_smem();
-          const uint32_t dst = sb + kBOffKv + buf * kBKvBytes;
-          const uint32_t bar = bars + 8 * (kBbKvFull + buf);
+          dst = sb + kBOffKv + buf * kBKvBytes;
+          bar = bars + 8 * (kBbKvFull + buf);
           mbar_arrive_expect_tx(bar, static_cast<uint32_t>(kBKvBytes));
+          ++uses;
+          return true;
+        };
+        int y = static_cast<int>(w.s.slot_off) + w.ti * kTile;
+        for (int k = 0; k < 2 * n_cache; ++k) {                 // cache tiles
+          uint32_t dst, bar;
+          if (!ring_slot(dst, bar)) { ok = false; break; }
           const CUtensorMap* map = (k & 1) ? &map_v : &map_k;
           tma_load_3d(dst, map, bar, 0, y, w.h);
           tma_load_3d(dst + kBHalf, map, bar, 64, y, w.h);
-          ++uses;
           y += (k & 1) * kTile;
         }
         if (!ok) break;
-        if (n_run > 0) {
-          w.ti += n_run - 1;            // bwalk_next moves past the run's last tile (and on to the next item)
-          w.it += n_run - 1;
-          w.piece_j += n_run - 1;
-          bwalk_next(a, w, pre);
-          continue;
+        int z = w.s.r0 + (w.ti + n_cache - ct) * kTile;
+        for (int k = 0; k < 2 * (n_run - n_cache); ++k) {       // the block's own key tiles
+          uint32_t dst, bar;
+          if (!ring_slot(dst, bar)) { ok = false; break; }
+          const CUtensorMap* map = (k & 1) ? &map_vs : &map_ks;
+          tma_load_3d(dst, map, bar, 0, w.h, z);
+          tma_load_3d(dst + kBHalf, map, bar, 64, w.h, z);
+          z += (k & 1) * kTile;
         }
+        if (!ok) break;
+        w.ti += n_run - 1;            // bwalk_next moves past the item's last tile and on to the next item
+        w.it += n_run - 1;
+        w.piece_j += n_run - 1;
+        bwalk_next(a, w, pre);
+        continue;
       }
       bwalk_tile(w);
       if (w.first) {
@@ -391,9 +412,11 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
     ok = issue_qk();
     while (ok && wp.it < n_iter) {
       // ---- a run of plain tiles needs neither walker: S of a tile that is neither the first nor the
-      //      last of its item, O += P V of a full cache tile that is not the first
+      //      last of its item, O += P V of a tile with all 128 keys valid that is not the first
       if (wq.item == wp.item && wp.ti > wp.ti_lo && wq.it == wp.it + 1) {
-        int n_run = min(wq.ti_hi - 1 - wq.ti, wp.s.L / kTile - wp.ti);
+        const int ct = wp.s.cache_tiles;
+        const int p_stop = wp.ti < ct ? wp.s.L / kTile : ct + wp.s.n_q / kTile;   // tiles with all 128 keys valid
+        int n_run = min(wq.ti_hi - 1 - wq.ti, p_stop - wp.ti);
         int it = wp.it;
         for (; n_run > 0; --n_run, ++it) {
           // S(it + 1)
@@ -603,10 +626,12 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
       return true;
     };
     while (ok && w.it < n_iter) {
-      // ---- a run of plain tiles -- full cache tiles that neither open nor close the item -- needs
-      //      none of the walker: most tiles of a long cache go through this loop
+      // ---- a run of plain tiles -- full cache tiles and step-local tiles left of the diagonal that
+      //      neither open nor close the item -- needs none of the walker nor a mask: most tiles of a
+      //      long cache or a long block go through this loop
       if (w.ti > w.ti_lo) {
-        const int stop = min(w.s.L / kTile, w.ti_hi - 1);
+        const int ct = w.s.cache_tiles;
+        const int stop = min(w.ti_hi - 1, w.ti < ct ? w.s.L / kTile : ct + big_plain_step_tiles(a, w.s, w.rt, tpt));
         while (w.ti < stop) {
           const int it = w.it;
           if (!wait_all(bar_s_full(it), (it >> 1) & 1) ||
@@ -640,7 +665,8 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
       {
         const int nv = w.nvalid;
         const bool is_step = w.step_idx >= 0;
-        if (!tile_body(is_step || nv < kTile, w.piece_j == 0, nv, is_step, w.step_idx, it)) { ok = false; break; }
+        const bool masked = is_step ? (w.step_idx >= big_plain_step_tiles(a, w.s, w.rt, tpt)) : (nv < kTile);
+        if (!tile_body(masked, w.piece_j == 0, nv, is_step, w.step_idx, it)) { ok = false; break; }
       }
 
       if (w.last) {
