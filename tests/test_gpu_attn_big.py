@@ -91,3 +91,14 @@ def test_prefill_sized_blocks():
     # behind an already cached part, for two sequences of different length
     check_attn(random_problem(2, 8, 2, 128, [0, 0], [1500, 700], [1500, 700], seed=51), "prefill, empty cache")
     check_attn(random_problem(2, 8, 2, 128, [1000, 3], [1024, 257], [1024, 257], seed=52), "chunked prefill")
+
+
+def test_long_blocks_whose_key_tiles_left_of_the_diagonal_still_need_the_mask():
+    # A long block's key tiles left of the diagonal skip the mask only if all rows and keys there are
+    # candidates with default anchors.  Here they are not: foresight rows behind the candidates
+    # (they see the candidates up to their anchor and themselves, not each other), custom anchors.
+    check_attn(random_problem(2, 8, 2, 128, [300, 0], [400, 300], [350, 300], seed=53),
+               "foresight rows behind a long run of candidates")
+    check_attn(random_problem(2, 8, 2, 128, [129, 0], [400, 300], [350, 260], seed=54, anchors=True),
+               "long blocks with custom anchors")
+    check_attn(random_problem(1, 4, 1, 128, [0], [640], [640], seed=55), "all candidates, G = 4, one head")
