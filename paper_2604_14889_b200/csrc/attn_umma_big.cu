@@ -207,6 +207,17 @@ __device__ __forceinline__ void big_load_scores(uint32_t s_addr, float (&v)[kBCw
     v[e] = s;
   }
 }
+// The same when the visible keys of the row are a prefix of the warpgroup's columns (a ragged cache
+// tile; a causal tile of a block whose rows are all candidates): columns from `limit` on become -inf.
+__device__ __forceinline__ void big_load_scores_prefix(uint32_t s_addr, float (&v)[kBCw], int limit) {
+  uint32_t raw[kBCw / 32][32];
+#pragma unroll
+  for (int c = 0; c < kBCw / 32; ++c) tmem_ld32(s_addr + c * 32, raw[c]);
+#pragma unroll
+  for (int c = 0; c < kBCw / 32; ++c) tmem_ld_wait(raw[c]);
+#pragma unroll
+  for (int e = 0; e < kBCw; ++e) v[e] = (e < limit) ? __uint_as_float(raw[e >> 5][e & 31]) : -INFINITY;
+}
 __device__ __forceinline__ float max_cols(const float (&v)[kBCw]) {
   float m[8];
 #pragma unroll
@@ -554,10 +565,15 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
       const uint32_t s_addr = lane_addr + kBColS + pb * kTile + wg * kBCw;
       const int key0 = (is_step ? step_idx * kTile : 0) + wg * kBCw;   // step-local index of column 0
       float v[kBCw];
-      if (masked)
-        big_load_scores<true>(s_addr, v, wg * kBCw, nv, is_step, tok, key0, w.s.n_c, anc,
-                              a.tok_kind ? a.tok_kind + w.s.r0 : nullptr, a.tok_kind ? a.tok_step + w.s.r0 : nullptr);
-      else
+      if (masked) {
+        // causal block of candidates only (prefill, compression): row `tok` sees the keys up to itself
+        const bool causal = !a.tok_kind && !a.anchor && min(w.s.n_q, (w.rt + 1) * tpt) <= w.s.n_c;
+        if (!is_step || causal)
+          big_load_scores_prefix(s_addr, v, (is_step ? min(nv, tok - step_idx * kTile + 1) : nv) - wg * kBCw);
+        else
+          big_load_scores<true>(s_addr, v, wg * kBCw, nv, is_step, tok, key0, w.s.n_c, anc,
+                                a.tok_kind ? a.tok_kind + w.s.r0 : nullptr, a.tok_kind ? a.tok_step + w.s.r0 : nullptr);
+      } else
         big_load_scores<false>(s_addr, v, 0, kTile, false, 0, 0, 0, 0);
       if (opens_item) {
         // new unit: reference = exact maximum of the first tile over all column groups
