@@ -395,23 +395,22 @@ def main():
         a_.record()
         b_.record()
 
-    def attn_params(ev=None, q=q_work, ks=ks_work):
-        return ms.attn_params(
-            batch=B, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, k_cache=inp.k_cache[0], v_cache=inp.v_cache[0],
-            kv_head_stride=stride, n_slots=inp.n_slots, kv_off=inp.kv_off, kv_len=inp.kv_len, max_kv_len=max_kv,
-            max_nq=nq, q_off=inp.q_off, n_cand=inp.n_cand, anchor=None, total_rows=T, sm_scale=0.0, q=q, k_step=ks,
-            v_step=inp.v_step, out=out, lse=lse, workspace=ws, workspace_bytes=wsb,
-            ev_split_begin=None if ev is None else ev[0].cuda_event,
-            ev_split_end=None if ev is None else ev[1].cuda_event)
-
-    plain = attn_params()
+    plain = ms.attn_params(
+        batch=B, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, k_cache=inp.k_cache[0], v_cache=inp.v_cache[0],
+        kv_head_stride=stride, n_slots=inp.n_slots, kv_off=inp.kv_off, kv_len=inp.kv_len, max_kv_len=max_kv,
+        max_nq=nq, q_off=inp.q_off, n_cand=inp.n_cand, anchor=None, total_rows=T, sm_scale=0.0, q=q_work,
+        k_step=ks_work, v_step=inp.v_step, out=out, lse=lse, workspace=ws, workspace_bytes=wsb)
 
     def step(s, ev=None):
         ms.memosight_rope_qk(q_work, ks_work, pos, T, Hq, Hkv, D, cfg.rope_base)
-        ms.memosight_attn_step(plain if ev is None else attn_params(ev))
+        if ev is not None:
+            ms.memosight_attn_debug_events(ev[0].cuda_event, ev[1].cuda_event)
+        ms.memosight_attn_step(plain)
+        if ev is not None:
+            ms.memosight_attn_debug_events(None, None)
         ms.memosight_accept(acc.logits, acc.ld_v, cfg.vocab, acc.row_off, B, T, acc.draft, am, nm, nk, aws, awb)
-        ms.memosight_kv_append(inp.k_cache[0], inp.v_cache[0], stride, B, Hkv, D, inp.kv_off, inp.kv_len, ks_work,
-                               inp.v_step, inp.q_off, inp.n_cand, nk, nq, 1)
+        ms.memosight_kv_append(inp.k_cache[0], inp.v_cache[0], stride, inp.n_slots, B, Hkv, D, inp.kv_off,
+                               inp.kv_len, None, ks_work, inp.v_step, inp.q_off, inp.n_cand, nk, nq, 1)
         ms.memosight_kv_compact(inp.k_cache, inp.v_cache, 1, Hkv * stride, stride, B, Hkv, D, inp.kv_off,
                                 inp.kv_len, seg_start[s], seg_len[s], None, 0, MEM_TOKENS + 1)
 
@@ -571,15 +570,17 @@ def run_compress(args, ms, dev, world, rank):
         seg_start.copy_(inp.kv_len)                  # the finished step starts where the cache ended ...
         inp.kv_len.add_(SEG_LEN)                     # ... and its 512 entries are in the cache
         ms.memosight_rope_qk(q_work, ks_work, pos, T, Hq, Hkv, D, cfg.rope_base)
+        if ev is not None:
+            ms.memosight_attn_debug_events(ev[0].cuda_event, ev[1].cuda_event)
         ms.memosight_attn_step(
             batch=B, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, k_cache=inp.k_cache[0], v_cache=inp.v_cache[0],
             kv_head_stride=stride, n_slots=inp.n_slots, kv_off=inp.kv_off, kv_len=inp.kv_len, max_kv_len=max_kv,
             max_nq=nq, q_off=inp.q_off, n_cand=inp.n_cand, anchor=None, total_rows=T, sm_scale=0.0, q=q_work,
-            k_step=ks_work, v_step=inp.v_step, out=out, lse=None, workspace=ws, workspace_bytes=wsb,
-            ev_split_begin=None if ev is None else ev[0].cuda_event,
-            ev_split_end=None if ev is None else ev[1].cuda_event)
-        ms.memosight_kv_append(inp.k_cache[0], inp.v_cache[0], stride, B, Hkv, D, inp.kv_off, inp.kv_len, ks_work,
-                               inp.v_step, inp.q_off, inp.n_cand, keep, nq, 1)
+            k_step=ks_work, v_step=inp.v_step, out=out, lse=None, workspace=ws, workspace_bytes=wsb)
+        if ev is not None:
+            ms.memosight_attn_debug_events(None, None)
+        ms.memosight_kv_append(inp.k_cache[0], inp.v_cache[0], stride, inp.n_slots, B, Hkv, D, inp.kv_off,
+                               inp.kv_len, None, ks_work, inp.v_step, inp.q_off, inp.n_cand, keep, nq, 1)
         ms.memosight_kv_compact(inp.k_cache, inp.v_cache, 1, Hkv * stride, stride, B, Hkv, D, inp.kv_off,
                                 inp.kv_len, seg_start, seg_len, None, 0, nq)
 

@@ -24,6 +24,11 @@
  *     the default stream), never synchronise, never allocate device memory and
  *     never read device scalars on the host: ragged lengths stay on the device
  *     and the caller supplies host-side upper bounds for launch sizing.
+ *   - the kernels are launched with programmatic stream serialisation: each may
+ *     begin its set-up while the kernel before it in the stream drains, and waits
+ *     for that kernel before it touches global memory, so stream order holds as usual.
+ *   - the first call of an entry point on a device sets that device up for it
+ *     (function attributes, symbol addresses): make it outside any stream capture.
  *   - return value: MS_OK or a negative MS_ERR_* code.  Arguments are validated
  *     on the host before anything is launched; a rejected call has no effect.
  *     Device code never traps; the only device-side failure (a bounded wait that
@@ -113,7 +118,9 @@ MS_API int32_t memosight_step_pids(int32_t p0, int32_t n_c, int32_t d, const int
  *   k       device bf16 [T][H_kv][D]  (may be NULL when H_kv == 0)
  *   pos_id  device int32 [T]
  *   inv_freq host double [D/2] or NULL; NULL means theta_i = rope_base^(-2i/D)
- * Angles and the rotation are evaluated in fp64 and rounded to bf16 once.
+ * The result of every element is the fp64 rotation (fp64 angle, fp64 sine and cosine) rounded
+ * to bf16 once; the kernel computes it in fp32 wherever that provably gives the same bits and in
+ * fp64 for the few elements next to a rounding boundary.
  * D even, 2 <= D <= 256.  T == 0 is a no-op. */
 MS_API int32_t memosight_rope_qk(void* q, void* k, const int32_t* pos_id, int32_t T, int32_t H_q,
                           int32_t H_kv, int32_t D, double rope_base, const double* inv_freq,
@@ -156,8 +163,6 @@ typedef struct memosight_attn_params {
   float* lse;                /* device fp32 [T][H_q], natural-log sum-exp, or NULL             */
   void* workspace;           /* device scratch, 256-byte aligned                               */
   size_t workspace_bytes;    /* >= memosight_attn_workspace_bytes(...)                         */
-  void* ev_split_begin;      /* optional cudaEvent_t recorded on `stream` right before ...     */
-  void* ev_split_end;        /* ... and right after the split-KV kernel (NULL: not recorded)   */
   /* Optional training-time mask (Sec. 2.3 "Attention Mask Strategy"), both or neither.  The block
    * is then an augmented sequence (Sec. 2.2) whose tokens carry a kind and a reasoning-step index;
    * among the block's own keys, key j is visible to row i iff j == i, or j < i and j is neither a
@@ -192,15 +197,40 @@ MS_API size_t memosight_attn_workspace_bytes(int32_t batch, int32_t n_q_heads, i
  * that overlap on the GPU need two workspaces. */
 MS_API int32_t memosight_attn_step(const memosight_attn_params* params, memosight_stream_t stream);
 
+/* The same attention for n_layers stacked layers that share the step's metadata (lengths, block
+ * offsets, candidates, anchors): Algorithm 1 forwards the whole model per step and keeps one
+ * cache per layer, all of the same length.  Layer l reads the cache at k_cache / v_cache +
+ * l * kv_layer_stride, the step tensors at q + l * q_layer_stride and k_step / v_step +
+ * l * kstep_layer_stride, and writes out + l * out_layer_stride (lse + l * lse_layer_stride);
+ * strides in elements, multiples of 8, each at least the size of one layer's tensor.  Step blocks
+ * of head_dim 128 with up to 64 packed rows run all layers in ONE launch of the keys-on-lanes
+ * kernel (the tile list is simply layer-major; tile prefix, workspace and tensor maps are shared);
+ * other shapes are issued layer by layer.  The workspace is the one memosight_attn_workspace_bytes
+ * gives for a single layer.  (A model that needs layer l's output before it can form layer l+1's
+ * queries calls memosight_attn_step per layer; this entry serves callers that hold every layer's
+ * q / k / v at once, and measures the stacked-layer step.) */
+typedef struct memosight_attn_layers {
+  uint32_t struct_size;        /* sizeof(memosight_attn_layers)                               */
+  int32_t n_layers;            /* >= 0; 1 behaves like memosight_attn_step                    */
+  int64_t kv_layer_stride;     /* elements between consecutive layers of k_cache / v_cache    */
+  int64_t q_layer_stride;      /* ... of q                                                    */
+  int64_t kstep_layer_stride;  /* ... of k_step and of v_step                                 */
+  int64_t out_layer_stride;    /* ... of out                                                  */
+  int64_t lse_layer_stride;    /* ... of lse (ignored when lse is NULL)                       */
+} memosight_attn_layers;
+MS_API int32_t memosight_attn_step_layers(const memosight_attn_params* params,
+                                          const memosight_attn_layers* layers, memosight_stream_t stream);
+
 /* Diagnostic switch: which kernel memosight_attn_step uses from now on, process-wide.
  * MS_ATTN_PATH_AUTO (the default) picks by shape: head_dim 128 with up to 64 packed rows
  * (max_nq * H_q/H_kv) takes the keys-on-lanes tcgen05 kernel, more rows or blocks of more than
  * 16 tokens the row-tiled large-block kernel; head_dim 64 the mma.sync kernel (up to 64 rows)
- * or the rows-on-lanes tcgen05 kernel (up to 128); anything else the general kernel.  Forcing a path that does not cover a shape falls back to the automatic choice for
- * that call (MS_ATTN_PATH_LARGE_BLOCK on a step block also needs a workspace of the size a
- * large-block call of the same bounds would get).  Returns the previous setting, or MS_ERR_INVALID_ARG.  Results of all paths agree
- * within the tolerance of bf16 inputs with fp32 accumulation; the switch exists for tests and
- * timing. */
+ * or the rows-on-lanes tcgen05 kernel (up to 128); anything else the general kernel.  A forced
+ * path is used only for calls whose shape it covers AND whose workspace is large enough for it
+ * (a path may need more than memosight_attn_workspace_bytes answers for the automatic choice);
+ * any other call falls back to the automatic choice.  Returns the previous setting, or
+ * MS_ERR_INVALID_ARG.  Results of all paths agree within the tolerance of bf16 inputs with fp32
+ * accumulation; the switch exists for tests and timing. */
 #define MS_ATTN_PATH_AUTO 0
 #define MS_ATTN_PATH_MMA_SYNC 1
 #define MS_ATTN_PATH_TCGEN05 2
@@ -208,6 +238,12 @@ MS_API int32_t memosight_attn_step(const memosight_attn_params* params, memosigh
 #define MS_ATTN_PATH_TCGEN05_KEYS 4   /* tcgen05 with the keys on the accumulator lanes; <= 64 rows, D 128 */
 #define MS_ATTN_PATH_LARGE_BLOCK 5    /* the row-tiled tcgen05 kernel of large blocks, for any block size; D 128 */
 MS_API int32_t memosight_attn_set_path(int32_t path);
+
+/* Diagnostic: from now on the attention calls of THIS thread record the two cudaEvent_t (passed
+ * as void*) on their stream right before and right after the split-KV kernel, so that a
+ * benchmark can time that kernel alone; (NULL, NULL) switches it off again.  Event records
+ * between the kernels keep a call from overlapping its launches, so leave it off otherwise. */
+MS_API int32_t memosight_attn_debug_events(void* ev_split_begin, void* ev_split_end);
 
 /* Synchronises `stream` and returns MS_OK, or MS_ERR_DEVICE_TIMEOUT if a kernel
  * of the last memosight_attn_step on this workspace gave up on a bounded wait
@@ -256,14 +292,21 @@ MS_API int32_t memosight_kv_gather(void* k_cache, void* v_cache, int32_t n_layer
 /* Appends the accepted candidates of each block to one layer's cache: the first
  * n_keep[b] rows of block b in k_step/v_step go to slots kv_len[b] .. of sequence
  * b.  n_keep[b] is clamped to [0, n_cand[b]]: a foresight row is never cached
- * (no later token may attend to it, Sec. 2.3).  kv_len[b] += n_keep[b] iff
- * bump_len != 0 (pass it on the last layer).  max_nq: host bound of block sizes.
- *   k_cache, v_cache device bf16 [H_kv][n_slots][D]; k_step, v_step device bf16 [T][H_kv][D] */
-MS_API int32_t memosight_kv_append(void* k_cache, void* v_cache, int64_t kv_head_stride, int32_t batch,
-                            int32_t n_kv_heads, int32_t head_dim, const int64_t* kv_off,
-                            int32_t* kv_len, const void* k_step, const void* v_step,
+ * (no later token may attend to it, Sec. 2.3).  It is clamped to the room the sequence has,
+ * too: to kv_cap[b] - kv_len[b] when kv_cap is given, and always to the end of the cache tensor
+ * (n_slots - kv_off[b] - kv_len[b]), so an append never writes into another sequence's slots or
+ * behind the tensor; when room, not the request, decided, *overflow is set to 1 (the caller
+ * clears it).  kv_len[b] += (what was appended) iff bump_len != 0 (pass it on the last layer; the
+ * clamps depend on kv_len, so every layer of a step appends the same rows).
+ *   k_cache, v_cache device bf16 [H_kv][n_slots][D]; k_step, v_step device bf16 [T][H_kv][D]
+ *   kv_cap   device int32 [B] or NULL: most entries sequence b may hold
+ *   overflow device int32 [1] or NULL
+ *   max_nq   host bound of the block sizes */
+MS_API int32_t memosight_kv_append(void* k_cache, void* v_cache, int64_t kv_head_stride, int64_t n_slots,
+                            int32_t batch, int32_t n_kv_heads, int32_t head_dim, const int64_t* kv_off,
+                            int32_t* kv_len, const int32_t* kv_cap, const void* k_step, const void* v_step,
                             const int32_t* q_off, const int32_t* n_cand, const int32_t* n_keep,
-                            int32_t max_nq, int32_t bump_len, memosight_stream_t stream);
+                            int32_t max_nq, int32_t bump_len, int32_t* overflow, memosight_stream_t stream);
 
 /* ---- Greedy accept (Sec. 2.1.1 and its footnote) ----------------------------------------- */
 
@@ -431,6 +474,7 @@ typedef struct memosight_step_host_params {
   const int32_t* d_seg_start;    /* device [B] or NULL: compaction request after the append    */
   const int32_t* d_seg_len;      /* device [B] (0 = skip sequence) when d_seg_start != NULL    */
   int32_t max_tail;              /* host bound of the entries a compaction moves               */
+  const int32_t* d_kv_cap;       /* device [B] or NULL: capacity of each sequence (kv_append)  */
   void* h_out;                   /* host bf16 [T][H_q][D]                                      */
   int32_t* h_argmax;             /* host [T] or NULL                                           */
   int32_t* h_n_match;            /* host [B] or NULL                                           */

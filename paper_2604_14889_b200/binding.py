@@ -65,8 +65,16 @@ class AttnParams(C.Structure):
         ("q", C.c_void_p), ("k_step", C.c_void_p), ("v_step", C.c_void_p),
         ("out", C.c_void_p), ("lse", C.c_void_p),
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
-        ("ev_split_begin", C.c_void_p), ("ev_split_end", C.c_void_p),
         ("tok_kind", C.c_void_p), ("tok_step", C.c_void_p),
+    ]
+
+
+class AttnLayers(C.Structure):
+    """Mirror of ``memosight_attn_layers`` (include/memosight.h)."""
+    _fields_ = [
+        ("struct_size", C.c_uint32), ("n_layers", C.c_int32), ("kv_layer_stride", C.c_int64),
+        ("q_layer_stride", C.c_int64), ("kstep_layer_stride", C.c_int64), ("out_layer_stride", C.c_int64),
+        ("lse_layer_stride", C.c_int64),
     ]
 
 
@@ -82,6 +90,7 @@ class StepHostParams(C.Structure):
         ("d_argmax", C.c_void_p), ("d_n_match", C.c_void_p), ("d_n_keep", C.c_void_p),
         ("accept_workspace", C.c_void_p), ("accept_workspace_bytes", C.c_size_t),
         ("d_seg_start", C.c_void_p), ("d_seg_len", C.c_void_p), ("max_tail", C.c_int32),
+        ("d_kv_cap", C.c_void_p),
         ("h_out", C.c_void_p), ("h_argmax", C.c_void_p), ("h_n_match", C.c_void_p),
     ]
 
@@ -129,6 +138,10 @@ def lib() -> C.CDLL:
         L.memosight_attn_workspace_bytes.argtypes = [C.c_int32] * 6
         L.memosight_attn_step.restype = C.c_int32
         L.memosight_attn_step.argtypes = [C.POINTER(AttnParams), C.c_void_p]
+        L.memosight_attn_step_layers.restype = C.c_int32
+        L.memosight_attn_step_layers.argtypes = [C.POINTER(AttnParams), C.POINTER(AttnLayers), C.c_void_p]
+        L.memosight_attn_debug_events.restype = C.c_int32
+        L.memosight_attn_debug_events.argtypes = [C.c_void_p, C.c_void_p]
         L.memosight_attn_set_path.restype = C.c_int32
         L.memosight_attn_set_path.argtypes = [C.c_int32]
         L.memosight_attn_status.restype = C.c_int32
@@ -154,9 +167,10 @@ def lib() -> C.CDLL:
         L.memosight_decode_commit_compress.restype = C.c_int32
         L.memosight_decode_commit_compress.argtypes = [C.POINTER(DecodeState)] + [C.c_void_p] * 3
         L.memosight_kv_append.restype = C.c_int32
-        L.memosight_kv_append.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_int32, C.c_int32,
-                                          C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
-                                          C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p]
+        L.memosight_kv_append.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int32, C.c_int32,
+                                          C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                          C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p,
+                                          C.c_void_p]
         L.memosight_accept_workspace_bytes.restype = C.c_size_t
         L.memosight_accept_workspace_bytes.argtypes = [C.c_int32, C.c_int32]
         L.memosight_accept.restype = C.c_int32
@@ -257,8 +271,8 @@ def memosight_attn_workspace_bytes(batch: int, n_q_heads: int, n_kv_heads: int, 
 
 def attn_params(*, batch, n_q_heads, n_kv_heads, head_dim, k_cache, v_cache, kv_head_stride, n_slots,
                 kv_off, kv_len, max_kv_len, max_nq, q_off, n_cand, anchor, total_rows, sm_scale,
-                q, k_step, v_step, out, lse, workspace, workspace_bytes, ev_split_begin=None,
-                ev_split_end=None, tok_kind=None, tok_step=None) -> AttnParams:
+                q, k_step, v_step, out, lse, workspace, workspace_bytes, tok_kind=None,
+                tok_step=None) -> AttnParams:
     """Fills a memosight_attn_params structure (addresses only; nothing is copied)."""
     p = AttnParams()
     p.struct_size = C.sizeof(AttnParams)
@@ -272,7 +286,6 @@ def attn_params(*, batch, n_q_heads, n_kv_heads, head_dim, k_cache, v_cache, kv_
     p.q, p.k_step, p.v_step = _ptr(q), _ptr(k_step), _ptr(v_step)
     p.out, p.lse = _ptr(out), _ptr(lse)
     p.workspace, p.workspace_bytes = _ptr(workspace), workspace_bytes
-    p.ev_split_begin, p.ev_split_end = _ptr(ev_split_begin), _ptr(ev_split_end)
     p.tok_kind, p.tok_step = _ptr(tok_kind), _ptr(tok_step)
     return p
 
@@ -281,6 +294,26 @@ def memosight_attn_step(params: Optional[AttnParams] = None, stream=None, **fiel
     """memosight_attn_step(params) or memosight_attn_step(**fields of attn_params)."""
     p = params if params is not None else attn_params(**fields)
     _check(int(lib().memosight_attn_step(C.byref(p), _stream(stream))), "memosight_attn_step")
+
+
+def memosight_attn_step_layers(params: AttnParams, n_layers: int, kv_layer_stride: int, q_layer_stride: int,
+                               kstep_layer_stride: int, out_layer_stride: int, lse_layer_stride: int = 0,
+                               stream=None) -> None:
+    """The attention of n_layers stacked layers that share the step's metadata (strides in elements)."""
+    ly = AttnLayers()
+    ly.struct_size = C.sizeof(AttnLayers)
+    ly.n_layers = n_layers
+    ly.kv_layer_stride, ly.q_layer_stride = kv_layer_stride, q_layer_stride
+    ly.kstep_layer_stride, ly.out_layer_stride, ly.lse_layer_stride = kstep_layer_stride, out_layer_stride, lse_layer_stride
+    _check(int(lib().memosight_attn_step_layers(C.byref(params), C.byref(ly), _stream(stream))),
+           "memosight_attn_step_layers")
+
+
+def memosight_attn_debug_events(ev_split_begin=None, ev_split_end=None) -> None:
+    """Timing events (cudaEvent_t addresses) the calling thread's attention calls record around the
+    split-KV kernel; (None, None) switches it off."""
+    _check(int(lib().memosight_attn_debug_events(_ptr(ev_split_begin), _ptr(ev_split_end))),
+           "memosight_attn_debug_events")
 
 
 def memosight_step_host(params: StepHostParams, stream=None) -> None:
@@ -362,12 +395,14 @@ def memosight_kv_gather(k_cache, v_cache, n_layers, layer_stride, kv_head_stride
            "memosight_kv_gather")
 
 
-def memosight_kv_append(k_cache, v_cache, kv_head_stride, batch, n_kv_heads, head_dim, kv_off, kv_len, k_step,
-                        v_step, q_off, n_cand, n_keep, max_nq, bump_len, stream=None) -> None:
-    _check(int(lib().memosight_kv_append(_ptr(k_cache), _ptr(v_cache), kv_head_stride, batch, n_kv_heads,
-                                         head_dim, _ptr(kv_off), _ptr(kv_len), _ptr(k_step), _ptr(v_step),
-                                         _ptr(q_off), _ptr(n_cand), _ptr(n_keep), max_nq, int(bool(bump_len)),
-                                         _stream(stream))), "memosight_kv_append")
+def memosight_kv_append(k_cache, v_cache, kv_head_stride, n_slots, batch, n_kv_heads, head_dim, kv_off, kv_len,
+                        kv_cap, k_step, v_step, q_off, n_cand, n_keep, max_nq, bump_len, overflow=None,
+                        stream=None) -> None:
+    _check(int(lib().memosight_kv_append(_ptr(k_cache), _ptr(v_cache), kv_head_stride, n_slots, batch, n_kv_heads,
+                                         head_dim, _ptr(kv_off), _ptr(kv_len), _ptr(kv_cap), _ptr(k_step),
+                                         _ptr(v_step), _ptr(q_off), _ptr(n_cand), _ptr(n_keep), max_nq,
+                                         int(bool(bump_len)), _ptr(overflow), _stream(stream))),
+           "memosight_kv_append")
 
 
 def memosight_accept_workspace_bytes(total_rows: int, vocab: int) -> int:

@@ -8,9 +8,11 @@
 // a producer thread keeps six 32 KB bulk copies (cp.async.bulk, global -> shared
 // memory, completion on an mbarrier) in flight, six warps take a chunk each from
 // the ring and reduce it with shuffles only.  Other layouts fall back to one CTA per
-// (chunk, row) with plain loads.  Pass 2 uses one warp per sequence:
-// each lane folds the chunk candidates of one row, then lane 0 walks the block's
-// rows to count the matching prefix.  Ordering rule everywhere: a NaN beats any
+// (chunk, row) with plain loads.  Pass 2 folds the chunk candidates of every row and counts
+// the matching prefix of every sequence.  In the streaming form it needs no launch of its own:
+// the warp that delivers the last chunk of a row (one atomicAdd on a per-row counter that
+// started at zero) folds that row, and the warp that folds the last row of all counts the
+// prefixes -- nobody waits for anybody.  Ordering rule everywhere: a NaN beats any
 // number, larger value beats smaller, equal values (and two NaNs) go to the lower
 // index -- the lowest-index-of-the-maximum convention with NaN treated as maximal.
 #include <limits.h>
@@ -111,9 +113,80 @@ constexpr int kStreamSmem = kStages * kStageBytes + 2 * kStages * 8 + 16;
 // candidates of the chunks that were not finished then carry index -1, which matches no draft.
 static __device__ unsigned int g_accept_wait_status;
 
+// What pass 2 needs when it runs inside pass 1.  cnt: a zeroed counter per row and, at index T,
+// one for the rows that are complete (left at zero again); NULL: a second kernel does pass 2.
+struct Tail {
+  unsigned int* cnt;
+  const int32_t* row_off;
+  const int32_t* draft;
+  int32_t* argmax_out;
+  int32_t* n_match;
+  int32_t* n_keep;
+  int B, T;
+};
+
+__device__ __forceinline__ Cand load_cand(const Cand* p) {
+  const int2 raw = __ldcg(reinterpret_cast<const int2*>(p));
+  return Cand{__int_as_float(raw.x), raw.y};
+}
+
+// Longest prefix of the block's rows whose argmax equals the draft (no early exit, so that the
+// loads of a block are independent of one another).
+__device__ __forceinline__ int match_prefix(const int32_t* __restrict__ draft, const int32_t* argmax, int r0, int r1) {
+  int m = 0;
+  bool run = true;
+  for (int r = r0; r < r1; ++r) {
+    const int d = draft[r];
+    const int am = __ldcg(argmax + r);
+    run = run && d >= 0 && am == d;
+    m += run ? 1 : 0;
+  }
+  return m;
+}
+
+// Called by a whole warp after it has delivered `part[row * n_chunks + chunk]`.
+__device__ __forceinline__ void accept_tail(const Tail& t, const Cand* part, int n_chunks, int row, int lane) {
+  unsigned int prev = 0;
+  if (lane == 0) {
+    __threadfence();                                   // the candidate is visible before the count
+    prev = atomicAdd(t.cnt + row, 1u);
+  }
+  prev = __shfl_sync(0xffffffffu, prev, 0);
+  if (prev + 1u != static_cast<unsigned int>(n_chunks)) return;
+  // every chunk of this row is in: fold them
+  __threadfence();
+  Cand best{-INFINITY, INT_MAX};
+  const Cand* pr = part + static_cast<int64_t>(row) * n_chunks;
+  for (int c = lane; c < n_chunks; c += 32) {
+    const Cand x = load_cand(pr + c);
+    if (x.i < 0) { best.v = NAN; best.i = -1; }        // an unfinished chunk: the row matches no draft
+    else if (best.i != -1) fold(best, x.v, x.i);
+  }
+  const bool bad = __any_sync(0xffffffffu, best.i == -1);
+  best = warp_best(best);
+  unsigned int rows_done = 0;
+  if (lane == 0) {
+    t.argmax_out[row] = bad ? -1 : best.i;
+    t.cnt[row] = 0u;
+    __threadfence();
+    rows_done = atomicAdd(t.cnt + t.T, 1u);
+  }
+  rows_done = __shfl_sync(0xffffffffu, rows_done, 0);
+  if (rows_done + 1u != static_cast<unsigned int>(t.T)) return;
+  // every row has its argmax: the prefix of every sequence
+  __threadfence();
+  for (int b = lane; b < t.B; b += 32) {
+    const int r0 = t.row_off[b], r1 = t.row_off[b + 1];
+    const int m = match_prefix(t.draft, t.argmax_out, r0, r1);
+    t.n_match[b] = m;
+    if (t.n_keep) t.n_keep[b] = (r1 > r0) ? m + 1 : 0;
+  }
+  if (lane == 0) t.cnt[t.T] = 0u;
+}
+
 __global__ void __launch_bounds__(kStreamThreads, 1)
 argmax_stream_kernel(const float* __restrict__ logits, int64_t ld_v, int V, int n_chunks, int n_items,
-                     Cand* __restrict__ part) {
+                     Cand* __restrict__ part, const Tail tail) {
   extern __shared__ __align__(1024) uint8_t smem[];
   const uint32_t sb = ms::smem_u32(smem);
   const uint32_t bars = sb + kStages * kStageBytes;           // full[kStages], empty[kStages]
@@ -128,6 +201,8 @@ argmax_stream_kernel(const float* __restrict__ logits, int64_t ld_v, int V, int 
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
+  ms::pdl_wait();
+  ms::pdl_trigger();
   // this CTA's items: blockIdx.x, blockIdx.x + gridDim.x, ...  (item = row * n_chunks + chunk)
   const int n_local = (n_items - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) /
                       static_cast<int>(gridDim.x);
@@ -226,6 +301,7 @@ argmax_stream_kernel(const float* __restrict__ logits, int64_t ld_v, int V, int 
       best.i = -1;
     }
     if (lane == 0) part[item] = best;
+    if (tail.cnt) accept_tail(tail, part, n_chunks, row, lane);
   }
 }
 
@@ -233,6 +309,8 @@ __global__ void __launch_bounds__(128)
 accept_rows_kernel(const Cand* __restrict__ part, int n_chunks, const int32_t* __restrict__ row_off,
                    int B, const int32_t* __restrict__ draft, int32_t* __restrict__ argmax_out,
                    int32_t* __restrict__ n_match, int32_t* __restrict__ n_keep) {
+  ms::pdl_wait();
+  ms::pdl_trigger();
   const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (b >= B) return;
@@ -264,31 +342,47 @@ accept_rows_kernel(const Cand* __restrict__ part, int n_chunks, const int32_t* _
 }
 
 inline int chunks_of(int V) { return (V + kChunk - 1) / kChunk; }
+constexpr int kTailMaxBatch = 2048;   // beyond it one warp counting every sequence's prefix would be the long pole
 
-// Pass 1 in whichever form the layout allows.
-int32_t launch_pass1(const float* logits, int64_t ld_v, int vocab, int total_rows, Cand* part, cudaStream_t st) {
+// Both passes.  The streaming form of pass 1 carries pass 2 in its tail when a counter bank is to
+// be had and the problem fits it; otherwise, and for the other layouts, pass 2 is a second launch.
+int32_t launch_accept(const float* logits, int64_t ld_v, int vocab, const int32_t* row_off, int batch,
+                      int total_rows, const int32_t* draft, int32_t* argmax_out, int32_t* n_match,
+                      int32_t* n_keep, Cand* part, cudaStream_t st) {
   const int n_chunks = chunks_of(vocab);
   const int n_items = n_chunks * total_rows;
   const bool vec = ms::aligned16(logits) && (ld_v % 4 == 0);
-  if (vec && vocab % 4 == 0) {
-    static bool configured[64] = {false};
-    int dev = 0;
-    MS_CUDA_TRY(cudaGetDevice(&dev));
-    if (dev >= 0 && dev < 64 && !configured[dev]) {
-      MS_CUDA_TRY(cudaFuncSetAttribute(argmax_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       kStreamSmem));
-      configured[dev] = true;
+  Tail tail;
+  tail.cnt = nullptr;
+  tail.row_off = row_off; tail.draft = draft; tail.argmax_out = argmax_out;
+  tail.n_match = n_match; tail.n_keep = n_keep; tail.B = batch; tail.T = total_rows;
+  if (total_rows > 0) {
+    if (vec && vocab % 4 == 0) {
+      static bool configured[64] = {false};
+      int dev = 0;
+      MS_CUDA_TRY(cudaGetDevice(&dev));
+      if (dev >= 0 && dev < 64 && !configured[dev]) {
+        MS_CUDA_TRY(cudaFuncSetAttribute(argmax_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         kStreamSmem));
+        configured[dev] = true;
+      }
+      const int sms = ms::sm_count();
+      if (sms <= 0) return ms::cuda_status(cudaErrorNoDevice);
+      if (total_rows < ms::kDoneBankWords && batch <= kTailMaxBatch) tail.cnt = ms::done_bank(part);
+      MS_CUDA_TRY(ms::launch_pdl(argmax_stream_kernel, dim3(n_items < sms ? n_items : sms), dim3(kStreamThreads),
+                                 kStreamSmem, st, logits, ld_v, vocab, n_chunks, n_items, part, tail));
+      if (tail.cnt) return MS_OK;
+    } else if (vec) {
+      argmax_chunks_kernel<true><<<static_cast<unsigned>(n_items), kThreads, 0, st>>>(logits, ld_v, vocab, n_chunks, part);
+      MS_LAUNCH_CHECK();
+    } else {
+      argmax_chunks_kernel<false><<<static_cast<unsigned>(n_items), kThreads, 0, st>>>(logits, ld_v, vocab, n_chunks, part);
+      MS_LAUNCH_CHECK();
     }
-    const int sms = ms::sm_count();
-    if (sms <= 0) return ms::cuda_status(cudaErrorNoDevice);
-    argmax_stream_kernel<<<n_items < sms ? n_items : sms, kStreamThreads, kStreamSmem, st>>>(
-        logits, ld_v, vocab, n_chunks, n_items, part);
-  } else if (vec) {
-    argmax_chunks_kernel<true><<<static_cast<unsigned>(n_items), kThreads, 0, st>>>(logits, ld_v, vocab, n_chunks, part);
-  } else {
-    argmax_chunks_kernel<false><<<static_cast<unsigned>(n_items), kThreads, 0, st>>>(logits, ld_v, vocab, n_chunks, part);
   }
-  MS_LAUNCH_CHECK();
+  MS_CUDA_TRY(ms::launch_pdl(accept_rows_kernel, dim3((batch + 3) / 4), dim3(128), 0, st,
+                             static_cast<const Cand*>(part), n_chunks, row_off, batch, draft, argmax_out, n_match,
+                             n_keep));
   return MS_OK;
 }
 
@@ -315,16 +409,8 @@ extern "C" int32_t memosight_accept(const float* logits, int64_t ld_v, int32_t v
     return MS_ERR_WORKSPACE_TOO_SMALL;
   if (reinterpret_cast<uintptr_t>(workspace) & 7u) return MS_ERR_ALIGNMENT;
   cudaStream_t st = ms::as_stream(stream);
-  const int n_chunks = chunks_of(vocab);
   Cand* part = static_cast<Cand*>(workspace);
-  if (total_rows > 0) {
-    const int32_t rc1 = launch_pass1(logits, ld_v, vocab, total_rows, part, st);
-    if (rc1 != MS_OK) return rc1;
-  }
-  accept_rows_kernel<<<(batch + 3) / 4, 128, 0, st>>>(part, n_chunks, row_off, batch, draft,
-                                                      argmax_out, n_match, n_keep);
-  MS_LAUNCH_CHECK();
-  return MS_OK;
+  return launch_accept(logits, ld_v, vocab, row_off, batch, total_rows, draft, argmax_out, n_match, n_keep, part, st);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -382,12 +468,5 @@ extern "C" int32_t memosight_accept_static(const float* logits, int64_t ld_v, in
   cudaStream_t st = ms::as_stream(stream);
   // Nothing in the array has to start at zero: pass 1 writes every (row, chunk) entry that pass 2
   // reads, so whatever an earlier call left behind is overwritten before it is looked at.
-  if (total_rows > 0) {
-    const int32_t rc1 = launch_pass1(logits, ld_v, vocab, total_rows, part, st);
-    if (rc1 != MS_OK) return rc1;
-  }
-  accept_rows_kernel<<<(batch + 3) / 4, 128, 0, st>>>(part, n_chunks, row_off, batch, draft,
-                                                      argmax_out, n_match, n_keep);
-  MS_LAUNCH_CHECK();
-  return MS_OK;
+  return launch_accept(logits, ld_v, vocab, row_off, batch, total_rows, draft, argmax_out, n_match, n_keep, part, st);
 }

@@ -29,6 +29,14 @@ struct AttnArgs {
   float scale_log2;   // softmax scale * log2(e): scores live in the exp2 domain
   int max_kv_len, max_nq;
   void* workspace;
+  // Stacked layers (keys-on-lanes kernel): layer l reads the cache at k_cache + l * kv_layer_stride
+  // and the step tensors / writes the results at their pointer + l * the tensor's layer stride
+  // (all in elements).  n_layers == 1 everywhere else.
+  int n_layers;
+  int64_t kv_layer_stride, q_layer_stride, kstep_layer_stride, out_layer_stride, lse_layer_stride;
+  // Counters of the in-kernel merge (two per persistent CTA, zero between launches), or NULL:
+  // the merge is then a launch of its own.
+  unsigned int* done;
   cudaEvent_t ev_split_begin, ev_split_end;   // optional timing events around the split kernel
 };
 

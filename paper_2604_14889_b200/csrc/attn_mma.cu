@@ -480,95 +480,38 @@ attn_split_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
 
 // ---------------------------------------------------------------- merge kernel
 
-// One CTA per (sequence, KV head) unit that was cut across CTAs of the split
-// kernel; one warp per packed row (grid: unit x groups of four rows).  The lanes
-// look up one piece each -- its slot and (m, l) -- and fold those with warp shuffles
-// into the row's maximum and normaliser; then every lane accumulates its D/32 output
-// columns over the pieces, whose slots and weights go round by shuffle.
+// The merge as a launch of its own (used when the split kernel does not merge in its tail): one
+// CTA per (layer, sequence, KV head) unit and group of four packed rows, one warp per packed row
+// (merge_row).  Units that lie inside one CTA of the split kernel were written by it: nothing to do.
 template <int D>
 __global__ void __launch_bounds__(128)
 attn_merge_kernel(const AttnArgs a, int rows_pad, int n_ctas) {
-  const int b = blockIdx.x / a.H_kv, h = blockIdx.x - b * a.H_kv;
+  pdl_wait();
+  pdl_trigger();
+  const int units_per_layer = a.B * a.H_kv;
+  const int layer = blockIdx.x / units_per_layer, bh = blockIdx.x - layer * units_per_layer;
+  const int b = bh / a.H_kv, h = bh - b * a.H_kv;
   const int* ws_pre = reinterpret_cast<const int*>(reinterpret_cast<const uint8_t*>(a.workspace) +
                                                    kWsHeaderBytes);
   const float* ws_slots = reinterpret_cast<const float*>(
       reinterpret_cast<const uint8_t*>(a.workspace) + kWsHeaderBytes + ws_prefix_bytes());
   const int tiles_b = ws_pre[b + 1] - ws_pre[b];
   if (tiles_b == 0) return;
-  const long long n_tiles = static_cast<long long>(ws_pre[a.B]) * a.H_kv;
-  const long long u0 = static_cast<long long>(ws_pre[b]) * a.H_kv + static_cast<long long>(h) * tiles_b;
-  const long long u1 = u0 + tiles_b;
-  // CTAs whose ranges [start(i), start(i+1)) intersect [u0, u1): start(i) = n_tiles*i/n_ctas
-  const int c_lo = static_cast<int>(((u0 + 1) * n_ctas - 1) / n_tiles);
-  const int c_hi = static_cast<int>((u1 * n_ctas - 1) / n_tiles);
-  if (c_lo == c_hi) return;                      // whole unit inside one CTA: already written
+  const long long per_layer = static_cast<long long>(ws_pre[a.B]) * a.H_kv;
+  const long long u0 = layer * per_layer + static_cast<long long>(ws_pre[b]) * a.H_kv +
+                       static_cast<long long>(h) * tiles_b;
+  CutUnit cu;
+  if (!cut_unit(per_layer * a.n_layers, n_ctas, u0, u0 + tiles_b, cu)) return;   // whole unit inside one CTA
   int L, n_q, r0;
   seq_shape(a, b, L, n_q, r0);
   const int rows = n_q * a.G;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int r = blockIdx.y * 4 + warp;           // this warp's packed row
   if (r >= rows) return;
-  const size_t slot_floats = ws_slot_floats(D, rows_pad);
-  constexpr int E = D / 32;
-  float M = -INFINITY, Lsum = 0.f, acc[E];
-#pragma unroll
-  for (int e = 0; e < E; ++e) acc[e] = 0.f;
-  // the pieces in groups of 32: lane j of a group looks its piece up (slot, m, l); the group's
-  // outputs are then accumulated relative to the running maximum M
-  for (int c0 = c_lo; c0 <= c_hi; c0 += 32) {
-    const int c = c0 + lane;
-    int slot = -1;
-    float m = -INFINITY, l = 0.f;
-    if (c <= c_hi) {
-      const long long s0 = n_tiles * c / n_ctas, s1 = n_tiles * (c + 1) / n_ctas;
-      if (s1 > s0) {                             // a CTA with tiles
-        slot = 2 * c + ((s0 >= u0) ? 0 : 1);
-        const float* sp = ws_slots + slot * slot_floats + static_cast<size_t>(rows_pad) * D;
-        m = sp[r];
-        l = sp[rows_pad + r];
-      }
-    }
-    float gm = m;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) gm = fmaxf(gm, __shfl_xor_sync(0xffffffffu, gm, o));
-    const float M_new = fmaxf(M, gm);
-    const float rescale = (M == -INFINITY) ? 0.f : exp2f(M - M_new);
-    const float w = (m == -INFINITY) ? 0.f : exp2f(m - M_new);
-    float lw = l * w;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) lw += __shfl_xor_sync(0xffffffffu, lw, o);
-    Lsum = Lsum * rescale + lw;
-#pragma unroll
-    for (int e = 0; e < E; ++e) acc[e] *= rescale;
-    M = M_new;
-    const int cnt = min(32, c_hi - c0 + 1);
-#pragma unroll 4
-    for (int k = 0; k < cnt; ++k) {
-      const int sk = __shfl_sync(0xffffffffu, slot, k);
-      const float wk = __shfl_sync(0xffffffffu, w, k);
-      if (sk < 0 || wk == 0.f) continue;
-      const float* po = ws_slots + sk * slot_floats + static_cast<size_t>(r) * D + lane * E;
-      if (E == 4) {
-        const float4 x = *reinterpret_cast<const float4*>(po);
-        acc[0] += wk * x.x;
-        acc[1] += wk * x.y;
-        acc[2] += wk * x.z;
-        acc[3] += wk * x.w;
-      } else {
-        const float2 x = *reinterpret_cast<const float2*>(po);
-        acc[0] += wk * x.x;
-        acc[1] += wk * x.y;
-      }
-    }
-  }
   const int i = r / a.G, g = r - i * a.G;
   const int64_t orow = static_cast<int64_t>(r0 + i) * a.H_q + h * a.G + g;
-  const float inv = 1.f / Lsum;
-  __nv_bfloat16* op = a.out + orow * D + lane * E;
-#pragma unroll
-  for (int e = 0; e < E; e += 2)
-    *reinterpret_cast<uint32_t*>(op + e) = pack_bf16(acc[e] * inv, acc[e + 1] * inv);
-  if (a.lse && lane == 0) a.lse[orow] = (M + log2f(Lsum)) * 0.69314718055994531f;
+  merge_row<D>(ws_slots, rows_pad, cu, r, lane, a.out + layer * a.out_layer_stride + orow * D,
+               a.lse ? a.lse + layer * a.lse_layer_stride + orow : nullptr);
 }
 
 // ---------------------------------------------------------------- host side
@@ -631,12 +574,11 @@ int32_t launch_attn_mma(const AttnArgs& a, cudaStream_t st) {
 }
 
 int32_t launch_attn_merge(const AttnArgs& a, cudaStream_t st, int rows_pad, int n_ctas) {
-  const dim3 grid(static_cast<unsigned>(a.B * a.H_kv), static_cast<unsigned>((rows_pad + 3) / 4));
+  const dim3 grid(static_cast<unsigned>(a.n_layers * a.B * a.H_kv), static_cast<unsigned>((rows_pad + 3) / 4));
   if (a.D == 128)
-    attn_merge_kernel<128><<<grid, 128, 0, st>>>(a, rows_pad, n_ctas);
+    MS_CUDA_TRY(launch_pdl(attn_merge_kernel<128>, grid, dim3(128), 0, st, a, rows_pad, n_ctas));
   else
-    attn_merge_kernel<64><<<grid, 128, 0, st>>>(a, rows_pad, n_ctas);
-  MS_LAUNCH_CHECK();
+    MS_CUDA_TRY(launch_pdl(attn_merge_kernel<64>, grid, dim3(128), 0, st, a, rows_pad, n_ctas));
   return MS_OK;
 }
 

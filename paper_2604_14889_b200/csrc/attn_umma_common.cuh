@@ -168,6 +168,7 @@ __device__ __forceinline__ float warp_max_f32(float v) {
 // Position in the CTA's range of the flat tile list.  Every role walks the list
 // on its own with this state, so no tile metadata travels through shared memory.
 struct Walk {
+  int layer;           // the list is layer-major: all units of layer 0, then layer 1, ...
   int b, h, ti, tiles_b, L, n_q, r0, n_c;
   long long slot_off;
   int it, n_iter;
@@ -186,7 +187,9 @@ __device__ __forceinline__ void walk_load_seq(const AttnArgs& a, Walk& w) {
   w.n_c = n_c < 0 ? 0 : (n_c > w.n_q ? w.n_q : n_c);
   w.slot_off = a.kv_off[w.b];
 }
-__device__ __forceinline__ void walk_init(const AttnArgs& a, Walk& w, int b0, long long rel, int n_iter) {
+__device__ __forceinline__ void walk_init(const AttnArgs& a, Walk& w, int b0, long long rel, int n_iter,
+                                          int layer0 = 0) {
+  w.layer = layer0;
   w.b = b0;
   walk_load_seq(a, w);
   w.h = static_cast<int>(rel / w.tiles_b);
@@ -221,10 +224,14 @@ __device__ __forceinline__ void walk_next(const AttnArgs& a, Walk& w) {
     if (++w.h == a.H_kv) {
       w.h = 0;
       if (w.it < w.n_iter) {
+        // tiles remain, so a sequence with tiles lies ahead: in this layer or at the start of the next
         do {
-          ++w.b;
+          if (++w.b == a.B) {
+            w.b = 0;
+            ++w.layer;
+          }
           walk_load_seq(a, w);
-        } while (w.tiles_b == 0 && w.b + 1 < a.B);
+        } while (w.tiles_b == 0 && w.layer < a.n_layers);
       }
     }
   }

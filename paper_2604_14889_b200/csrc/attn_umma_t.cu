@@ -89,33 +89,15 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
   int* ws_pre = reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(a.workspace) + kWsHeaderBytes);
   float* ws_slots = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(a.workspace) + kWsHeaderBytes +
                                              ws_prefix_bytes());
+  volatile int* last_flags = reinterpret_cast<volatile int*>(smem + lay.off_misc + kMiscScalars + 24);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (sb & 1023u) {
+    pdl_wait();
     if (threadIdx.x == 0) atomicExch(status, kTimeoutMagic + 1);
     return;
   }
 
-  // ---- schedule (the prefix lives where the buffers will be) ----
-  int* s_pre = reinterpret_cast<int*>(smem);
-  int* s_scratch = s_pre + a.B + 1;
-  build_tile_prefix(a, s_pre, s_scratch);
-  const long long n_tiles = static_cast<long long>(s_pre[a.B]) * a.H_kv;
-  const long long t0 = n_tiles * blockIdx.x / gridDim.x;
-  const long long t1 = n_tiles * (blockIdx.x + 1) / gridDim.x;
-  const int n_iter = static_cast<int>(t1 - t0);
-  if (blockIdx.x == 0) {
-    for (int i = threadIdx.x; i <= a.B; i += blockDim.x) ws_pre[i] = s_pre[i];
-  }
-  Walk w0;
-  w0.n_iter = 0;
-  if (n_iter > 0) {
-    int lo = 0, hi = a.B;
-    while (hi - lo > 1) {
-      const int mid = (lo + hi) >> 1;
-      if (static_cast<long long>(s_pre[mid]) * a.H_kv <= t0) lo = mid; else hi = mid;
-    }
-    walk_init(a, w0, lo, t0 - static_cast<long long>(s_pre[lo]) * a.H_kv, n_iter);
-  }
+  // ---- set-up that touches no global memory: barriers, tensor memory ----
   if (threadIdx.x == 0) {
     for (int i = 0; i < kTMaxKv; ++i) {
       mbar_init(bars + 8 * (kTbKvFull + i), 1);
@@ -136,7 +118,12 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
     grow_flags[1] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  __syncthreads();   // the prefix has been consumed
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                     smem_u32(tmem_slot)), "r"(kCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
   // Rows of the Q buffers past the box are never loaded; as B rows they only feed the padded
   // score columns, which must stay finite: clear them once.
   {
@@ -150,14 +137,36 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
     }
     fence_async_smem();
   }
-  if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
-                     smem_u32(tmem_slot)), "r"(kCols)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  // ---- from here on global memory is read: the grid before this one must have finished ----
+  pdl_wait();
+  pdl_trigger();
+
+  // ---- schedule (the prefix lives where the K/V ring will be) ----
+  int* s_pre = reinterpret_cast<int*>(smem + lay.off_kv);
+  int* s_scratch = s_pre + a.B + 1;
+  build_tile_prefix(a, s_pre, s_scratch);
+  const long long per_layer = static_cast<long long>(s_pre[a.B]) * a.H_kv;
+  const long long n_tiles = per_layer * a.n_layers;
+  const long long t0 = n_tiles * blockIdx.x / gridDim.x;
+  const long long t1 = n_tiles * (blockIdx.x + 1) / gridDim.x;
+  const int n_iter = static_cast<int>(t1 - t0);
+  if (blockIdx.x == 0 && !a.done) {
+    for (int i = threadIdx.x; i <= a.B; i += blockDim.x) ws_pre[i] = s_pre[i];
+  }
+  Walk w0;
+  w0.n_iter = 0;
+  if (n_iter > 0) {
+    const int layer0 = static_cast<int>(t0 / per_layer);
+    const long long rem = t0 - layer0 * per_layer;
+    int lo = 0, hi = a.B;
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (static_cast<long long>(s_pre[mid]) * a.H_kv <= rem) lo = mid; else hi = mid;
+    }
+    walk_init(a, w0, lo, rem - static_cast<long long>(s_pre[lo]) * a.H_kv, n_iter, layer0);
   }
   tc_fence_before();
-  __syncthreads();
+  __syncthreads();   // the prefix has been consumed; barriers, tensor memory and the Q padding are ready
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
@@ -181,8 +190,8 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
         mbar_arrive_expect_tx(bar, static_cast<uint32_t>(HALVES * lay.rows_box * 128));
 #pragma unroll
         for (int hf = 0; hf < HALVES; ++hf)
-          tma_load_3d(sb + lay.off_q + qb * lay.q_bytes + hf * lay.q_half, &map_q, bar, hf * 64, w.h * a.G,
-                      w.r0);
+          tma_load_4d(sb + lay.off_q + qb * lay.q_bytes + hf * lay.q_half, &map_q, bar, hf * 64, w.h * a.G,
+                      w.r0, w.layer);
         ++pieces;
       }
 #pragma unroll 1
@@ -200,13 +209,13 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
           mbar_arrive_expect_tx(bar, static_cast<uint32_t>(HALVES * kMaxNq * 128));
 #pragma unroll
           for (int hf = 0; hf < HALVES; ++hf)
-            tma_load_3d(dst + hf * kHalfStrideT, kv ? &map_vs : &map_ks, bar, hf * 64, w.h, w.r0);
+            tma_load_4d(dst + hf * kHalfStrideT, kv ? &map_vs : &map_ks, bar, hf * 64, w.h, w.r0, w.layer);
         } else {
           mbar_arrive_expect_tx(bar, static_cast<uint32_t>(kKvBytes));
           const int y = static_cast<int>(w.slot_off) + w.ti * kTile;
 #pragma unroll
           for (int hf = 0; hf < HALVES; ++hf)
-            tma_load_3d(dst + hf * kHalfStrideT, kv ? &map_v : &map_k, bar, hf * 64, y, w.h);
+            tma_load_4d(dst + hf * kHalfStrideT, kv ? &map_v : &map_k, bar, hf * 64, y, w.h, w.layer);
         }
         ++uses;
       }
@@ -493,14 +502,16 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
 #pragma unroll
         for (int c = 0; c < CW / 8; ++c) tmem_ld_wait8(o + c * 8);
         // thread t holds element d = t of every row
+        __nv_bfloat16* out_l = a.out + w.layer * a.out_layer_stride;
+        float* lse_l = a.lse ? a.lse + w.layer * a.lse_layer_stride : nullptr;
         if (w.slot < 0) {
           int i = c0 / a.G, g = c0 - i * a.G;
 #pragma unroll
           for (int j = 0; j < CW; ++j) {
             if (c0 + j < rows) {
               const int64_t orow = static_cast<int64_t>(w.r0 + i) * a.H_q + w.h * a.G + g;
-              a.out[orow * D + t] = __float2bfloat16_rn(__uint_as_float(o[j]) / l_row[j]);
-              if (a.lse && t == j) a.lse[orow] = (m_mine + log2f(l_row[j])) * 0.69314718055994531f;
+              out_l[orow * D + t] = __float2bfloat16_rn(__uint_as_float(o[j]) / l_row[j]);
+              if (lse_l && t == j) lse_l[orow] = (m_mine + log2f(l_row[j])) * 0.69314718055994531f;
             }
             if (++g == a.G) { g = 0; ++i; }
           }
@@ -514,6 +525,30 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
               if (t == j) {
                 sm[c0 + j] = m_mine;
                 sm[rows_pad + c0 + j] = l_row[j];
+              }
+            }
+          }
+          if (a.done) {
+            // The unit is cut across CTAs.  Each warpgroup of each of its CTAs counts itself once its
+            // half of the partial rows is out; the one that counts last merges that half (nobody waits).
+            __threadfence();
+            if (!wg_sync()) { ok = false; break; }
+            CutUnit cu;
+            const long long u0 = t0 + w.it - w.ti;
+            cut_unit(n_tiles, static_cast<int>(gridDim.x), u0, u0 + w.tiles_b, cu);
+            if (t == 0) {
+              unsigned int* cnt = a.done + 2 * cu.c_lo + wg;
+              const bool is_last = atomicAdd(cnt, 1u) + 1u == static_cast<unsigned int>(cut_pieces(cu));
+              if (is_last) *cnt = 0u;
+              last_flags[wg] = is_last ? 1 : 0;
+            }
+            if (!wg_sync()) { ok = false; break; }
+            if (last_flags[wg]) {
+              __threadfence();
+              for (int j = quad; j < CW && c0 + j < rows; j += 4) {
+                const int r = c0 + j, i = r / a.G, g = r - i * a.G;
+                const int64_t orow = static_cast<int64_t>(w.r0 + i) * a.H_q + w.h * a.G + g;
+                merge_row<D>(ws_slots, rows_pad, cu, r, lane, out_l + orow * D, lse_l ? lse_l + orow : nullptr);
               }
             }
           }
@@ -564,8 +599,8 @@ int32_t launch_t(const AttnArgs& a, cudaStream_t st, int rows_pad, int grid, con
     configured[dev] = true;
   }
   if (a.ev_split_begin) MS_CUDA_TRY(cudaEventRecord(a.ev_split_begin, st));
-  attn_umma_t_kernel<NP><<<grid, kTThreads, lay.total, st>>>(a, mk, mv, mks, mvs, mq, rows_pad, lay);
-  MS_LAUNCH_CHECK();
+  MS_CUDA_TRY(launch_pdl(attn_umma_t_kernel<NP>, dim3(grid), dim3(kTThreads), static_cast<size_t>(lay.total), st, a,
+                         mk, mv, mks, mvs, mq, rows_pad, lay));
   if (a.ev_split_end) MS_CUDA_TRY(cudaEventRecord(a.ev_split_end, st));
   return MS_OK;
 }
@@ -574,23 +609,31 @@ int32_t launch_t(const AttnArgs& a, cudaStream_t st, int rows_pad, int grid, con
 
 bool attn_umma_t_supports(int D, int G, int max_nq) { return D == 128 && max_nq <= kMaxNq && G * max_nq <= 64; }
 
-int32_t launch_attn_umma_t(const AttnArgs& a, cudaStream_t st) {
-  if (a.B == 0 || a.T == 0) return MS_OK;
+int32_t launch_attn_umma_t(const AttnArgs& a_in, cudaStream_t st) {
+  AttnArgs a = a_in;
+  if (a.B == 0 || a.T == 0 || a.n_layers == 0) return MS_OK;
   const int rows = a.max_nq * a.G;
   const int rows_pad = (rows + 15) & ~15;
   TLayout lay;
   if (!attn_umma_t_supports(a.D, a.G, a.max_nq) || !plan_t_layout(rows_pad, rows, &lay))
     return MS_ERR_UNSUPPORTED_SHAPE;
-  if (static_cast<int>((a.B + 1 + kTThreads) * sizeof(int)) > lay.off_misc) return MS_ERR_UNSUPPORTED_SHAPE;
+  if (static_cast<int>((a.B + 1 + kTThreads / 32) * sizeof(int)) > lay.n_kv * kKvBytes) return MS_ERR_UNSUPPORTED_SHAPE;
   const int grid = attn_mma_grid();
   if (grid <= 0) return cuda_status(cudaErrorNoDevice);
+  // the merge runs in the kernel's tail when a bank of counters is to be had (two per CTA)
+  a.done = (2 * grid <= kDoneBankWords) ? done_bank(a.workspace) : nullptr;
+  // one descriptor per tensor covers every layer (the layer is the outermost coordinate)
+  const uint64_t nl = static_cast<uint64_t>(a.n_layers);
+  const uint64_t kv_ls = nl > 1 ? a.kv_layer_stride : static_cast<uint64_t>(a.H_kv) * a.kv_head_stride;
+  const uint64_t q_ls = nl > 1 ? a.q_layer_stride : static_cast<uint64_t>(a.T) * a.H_q * a.D;
+  const uint64_t ks_ls = nl > 1 ? a.kstep_layer_stride : static_cast<uint64_t>(a.T) * a.H_kv * a.D;
   CUtensorMap mk, mv, mks, mvs, mq;
   const bool ok =
-      make_map(&mk, a.k_cache, a.D, static_cast<uint64_t>(a.n_slots), a.H_kv, a.D, a.kv_head_stride, kTile, 1) &&
-      make_map(&mv, a.v_cache, a.D, static_cast<uint64_t>(a.n_slots), a.H_kv, a.D, a.kv_head_stride, kTile, 1) &&
-      make_map(&mks, a.k_step, a.D, a.H_kv, a.T, a.D, static_cast<uint64_t>(a.H_kv) * a.D, 1, kMaxNq) &&
-      make_map(&mvs, a.v_step, a.D, a.H_kv, a.T, a.D, static_cast<uint64_t>(a.H_kv) * a.D, 1, kMaxNq) &&
-      make_map(&mq, a.q, a.D, a.H_q, a.T, a.D, static_cast<uint64_t>(a.H_q) * a.D, a.G, a.max_nq);
+      make_map4(&mk, a.k_cache, a.D, static_cast<uint64_t>(a.n_slots), a.H_kv, nl, a.D, a.kv_head_stride, kv_ls, kTile, 1) &&
+      make_map4(&mv, a.v_cache, a.D, static_cast<uint64_t>(a.n_slots), a.H_kv, nl, a.D, a.kv_head_stride, kv_ls, kTile, 1) &&
+      make_map4(&mks, a.k_step, a.D, a.H_kv, a.T, nl, a.D, static_cast<uint64_t>(a.H_kv) * a.D, ks_ls, 1, kMaxNq) &&
+      make_map4(&mvs, a.v_step, a.D, a.H_kv, a.T, nl, a.D, static_cast<uint64_t>(a.H_kv) * a.D, ks_ls, 1, kMaxNq) &&
+      make_map4(&mq, a.q, a.D, a.H_q, a.T, nl, a.D, static_cast<uint64_t>(a.H_q) * a.D, q_ls, a.G, a.max_nq);
   if (!ok) return cuda_status(cudaErrorInvalidValue);
   int32_t rc;
   switch (rows_pad) {
@@ -599,7 +642,7 @@ int32_t launch_attn_umma_t(const AttnArgs& a, cudaStream_t st) {
     case 48: rc = launch_t<48>(a, st, rows_pad, grid, lay, mk, mv, mks, mvs, mq); break;
     default: rc = launch_t<64>(a, st, rows_pad, grid, lay, mk, mv, mks, mvs, mq); break;
   }
-  if (rc != MS_OK) return rc;
+  if (rc != MS_OK || a.done) return rc;
   return launch_attn_merge(a, st, rows_pad, grid);
 }
 

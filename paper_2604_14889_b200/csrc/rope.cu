@@ -2,10 +2,13 @@
 // IDs (paper Sec. 2.1.2: the position layouts of memory and foresight tokens act
 // through RoPE, so each new token is rotated by its own PID, not by its cache slot).
 //
-// One CTA per token.  The D/2 angles of the token are evaluated once in fp64
-// (sincos of pos * theta_i), kept in shared memory and reused by all H_q + H_kv
-// heads; the rotation is done in fp64 and rounded to bf16 once, so the result
-// equals an fp64 reference up to the last-bit behaviour of sin/cos.
+// One CTA per (token, run of heads).  The D/2 angles of the token are evaluated in fp64
+// (sincos of pos * theta_i) and kept in shared memory as fp64 and fp32.  The result of
+// every element is the fp64 rotation rounded to bf16 once -- but it is computed in fp32
+// whenever that provably gives the same bits: the fp32 value carries an error bound, and
+// if both ends of the bound round to the same bf16 number, so does the exact value
+// (rounding is monotonic).  Only the few elements that sit next to a rounding boundary
+// (about one in a thousand) are redone in fp64.
 #include <math.h>
 
 #include "common.cuh"
@@ -43,15 +46,36 @@ __device__ __forceinline__ uint16_t f64_to_bf16_bits(double x) {
   return static_cast<uint16_t>((x < 0 ? 0x8000u : 0u) | out);
 }
 
-__device__ __forceinline__ double bf16_bits_to_f64(uint16_t h) {
-  return static_cast<double>(__uint_as_float(static_cast<uint32_t>(h) << 16));
+// a*c - b*s (sign = -1) or a*c + b*s (sign = +1), a and b exact bf16 values, rounded to bf16 once.
+__device__ __forceinline__ uint16_t rot_elem(float a, float b, float c32, float s32, double c64, double s64,
+                                             float sign) {
+  const float bs = b * s32;
+  const float r = fmaf(a, c32, sign * bs);
+  // |r - exact| <= (|a c| + |b s|) * 3 * 2^-24 (two rounded constants, one rounded product, one
+  // rounded sum) + denormal slack; 5 * 2^-24 leaves room for the rounding of the bound itself
+  const float e = (fabsf(a * c32) + fabsf(bs)) * 2.98e-7f + 1e-44f;
+  const __nv_bfloat16 lo = __float2bfloat16_rn(r - e), hi = __float2bfloat16_rn(r + e);
+  const uint16_t lo_b = *reinterpret_cast<const uint16_t*>(&lo), hi_b = *reinterpret_cast<const uint16_t*>(&hi);
+  if (lo_b == hi_b && r == r) return lo_b;
+  const double ad = static_cast<double>(a), bd = static_cast<double>(b);
+  return f64_to_bf16_bits(sign < 0.f ? ad * c64 - bd * s64 : ad * c64 + bd * s64);
 }
 
-__global__ void __launch_bounds__(128)
+__device__ __forceinline__ float bf16_bits_to_f32(uint16_t h) {
+  return __uint_as_float(static_cast<uint32_t>(h) << 16);
+}
+
+constexpr int kRopeThreads = 128;
+
+__global__ void __launch_bounds__(kRopeThreads)
 rope_qk_kernel(uint16_t* __restrict__ q, uint16_t* __restrict__ k, const int32_t* __restrict__ pos_id,
-               int H_q, int H_kv, int D, uint32_t flags, bool vec_ok, FreqTable freq) {
+               int H_q, int H_kv, int D, int heads_per_cta, uint32_t flags, bool vec_ok, FreqTable freq) {
   __shared__ double s_cos[kMaxHalf];
   __shared__ double s_sin[kMaxHalf];
+  __shared__ float s_cos32[kMaxHalf];
+  __shared__ float s_sin32[kMaxHalf];
+  ms::pdl_wait();
+  ms::pdl_trigger();
   const int t = blockIdx.x;
   const int half = D >> 1;
   double p = static_cast<double>(pos_id[t]);
@@ -61,31 +85,34 @@ rope_qk_kernel(uint16_t* __restrict__ q, uint16_t* __restrict__ k, const int32_t
     sincos(p * freq.f[i], &s, &c);
     s_cos[i] = c;
     s_sin[i] = s;
+    s_cos32[i] = static_cast<float>(c);
+    s_sin32[i] = static_cast<float>(s);
   }
   __syncthreads();
   const bool interleaved = (flags & MS_ROPE_INTERLEAVED) != 0;
   const int n_heads = H_q + H_kv;
+  const int h_lo = blockIdx.y * heads_per_cta;
+  const int n_mine = min(heads_per_cta, n_heads - h_lo);
   if (vec_ok && (half & 7) == 0) {
     // 16-byte accesses: a work item is 8 consecutive pair indices of one head (rotate-half: 8
     // elements of each half) or 4 of them (interleaved: 8 consecutive elements)
     const int per_head = interleaved ? half / 4 : half / 8;
-    for (int w = threadIdx.x; w < n_heads * per_head; w += blockDim.x) {
-      const int h = w / per_head, c = w - h * per_head;
+    for (int w = threadIdx.x; w < n_mine * per_head; w += blockDim.x) {
+      const int hh = w / per_head, c = w - hh * per_head, h = h_lo + hh;
       uint16_t* v = (h < H_q) ? q + (static_cast<int64_t>(t) * H_q + h) * D
                               : k + (static_cast<int64_t>(t) * H_kv + (h - H_q)) * D;
       if (interleaved) {
-        uint4* p = reinterpret_cast<uint4*>(v + 8 * c);
-        uint4 x = *p;
+        uint4* pv = reinterpret_cast<uint4*>(v + 8 * c);
+        uint4 x = *pv;
         uint16_t* e = reinterpret_cast<uint16_t*>(&x);
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           const int i = 4 * c + j;
-          const double a = bf16_bits_to_f64(e[2 * j]), b = bf16_bits_to_f64(e[2 * j + 1]);
-          const double cs = s_cos[i], sn = s_sin[i];
-          e[2 * j] = f64_to_bf16_bits(a * cs - b * sn);
-          e[2 * j + 1] = f64_to_bf16_bits(b * cs + a * sn);
+          const float a = bf16_bits_to_f32(e[2 * j]), b = bf16_bits_to_f32(e[2 * j + 1]);
+          e[2 * j] = rot_elem(a, b, s_cos32[i], s_sin32[i], s_cos[i], s_sin[i], -1.f);
+          e[2 * j + 1] = rot_elem(b, a, s_cos32[i], s_sin32[i], s_cos[i], s_sin[i], 1.f);
         }
-        *p = x;
+        *pv = x;
       } else {
         uint4* pa = reinterpret_cast<uint4*>(v + 8 * c);
         uint4* pb = reinterpret_cast<uint4*>(v + half + 8 * c);
@@ -95,10 +122,9 @@ rope_qk_kernel(uint16_t* __restrict__ q, uint16_t* __restrict__ k, const int32_t
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
           const int i = 8 * c + j;
-          const double a = bf16_bits_to_f64(ea[j]), b = bf16_bits_to_f64(eb[j]);
-          const double cs = s_cos[i], sn = s_sin[i];
-          ea[j] = f64_to_bf16_bits(a * cs - b * sn);
-          eb[j] = f64_to_bf16_bits(b * cs + a * sn);
+          const float a = bf16_bits_to_f32(ea[j]), b = bf16_bits_to_f32(eb[j]);
+          ea[j] = rot_elem(a, b, s_cos32[i], s_sin32[i], s_cos[i], s_sin[i], -1.f);
+          eb[j] = rot_elem(b, a, s_cos32[i], s_sin32[i], s_cos[i], s_sin[i], 1.f);
         }
         *pa = xa;
         *pb = xb;
@@ -106,16 +132,15 @@ rope_qk_kernel(uint16_t* __restrict__ q, uint16_t* __restrict__ k, const int32_t
     }
     return;
   }
-  for (int w = threadIdx.x; w < n_heads * half; w += blockDim.x) {
-    const int h = w / half, i = w - h * half;
+  for (int w = threadIdx.x; w < n_mine * half; w += blockDim.x) {
+    const int hh = w / half, i = w - hh * half, h = h_lo + hh;
     uint16_t* v = (h < H_q) ? q + (static_cast<int64_t>(t) * H_q + h) * D
                             : k + (static_cast<int64_t>(t) * H_kv + (h - H_q)) * D;
     const int ia = interleaved ? 2 * i : i;
     const int ib = interleaved ? 2 * i + 1 : i + half;
-    const double a = bf16_bits_to_f64(v[ia]), b = bf16_bits_to_f64(v[ib]);
-    const double c = s_cos[i], s = s_sin[i];
-    v[ia] = f64_to_bf16_bits(a * c - b * s);
-    v[ib] = f64_to_bf16_bits(b * c + a * s);
+    const float a = bf16_bits_to_f32(v[ia]), b = bf16_bits_to_f32(v[ib]);
+    v[ia] = rot_elem(a, b, s_cos32[i], s_sin32[i], s_cos[i], s_sin[i], -1.f);
+    v[ib] = rot_elem(b, a, s_cos32[i], s_sin32[i], s_cos[i], s_sin[i], 1.f);
   }
 }
 
@@ -136,9 +161,14 @@ extern "C" int32_t memosight_rope_qk(void* q, void* k, const int32_t* pos_id, in
     freq.f[i] = inv_freq ? inv_freq[i] : pow(rope_base, -2.0 * static_cast<double>(i) / D);
   for (int i = D / 2; i < kMaxHalf; ++i) freq.f[i] = 0.0;
   const bool vec_ok = ms::aligned16(q) && ms::aligned16(k);   // NULL (no heads of that kind) counts as aligned
-  rope_qk_kernel<<<T, 128, 0, ms::as_stream(stream)>>>(static_cast<uint16_t*>(q),
-                                                        static_cast<uint16_t*>(k), pos_id, H_q, H_kv,
-                                                        D, flags, vec_ok, freq);
-  MS_LAUNCH_CHECK();
+  // few tokens: spread each token's heads over several CTAs (latency); many: one CTA per token, so
+  // that the fp64 angles are evaluated once
+  const int n_heads = H_q + H_kv;
+  const int heads_per_cta = T >= 2048 ? n_heads : (n_heads < 8 ? n_heads : 8);
+  const int chunks = (n_heads + heads_per_cta - 1) / heads_per_cta;
+  if (chunks > 65535) return MS_ERR_UNSUPPORTED_SHAPE;
+  MS_CUDA_TRY(ms::launch_pdl(rope_qk_kernel, dim3(T, chunks), dim3(kRopeThreads), 0, ms::as_stream(stream),
+                             static_cast<uint16_t*>(q), static_cast<uint16_t*>(k), pos_id, H_q, H_kv, D,
+                             heads_per_cta, flags, vec_ok, freq));
   return MS_OK;
 }

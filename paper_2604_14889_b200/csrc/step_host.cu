@@ -91,9 +91,9 @@ extern "C" int32_t memosight_step_host(const memosight_step_host_params* p,
                           stream);
     if (rc != MS_OK) return rc;
     rc = memosight_kv_append(const_cast<void*>(a.k_cache), const_cast<void*>(a.v_cache),
-                             a.kv_head_stride, B, a.n_kv_heads, a.head_dim, a.kv_off,
-                             const_cast<int32_t*>(a.kv_len), a.k_step, a.v_step, a.q_off, a.n_cand,
-                             p->d_n_keep, a.max_nq, 1, stream);
+                             a.kv_head_stride, a.n_slots, B, a.n_kv_heads, a.head_dim, a.kv_off,
+                             const_cast<int32_t*>(a.kv_len), p->d_kv_cap, a.k_step, a.v_step, a.q_off,
+                             a.n_cand, p->d_n_keep, a.max_nq, 1, nullptr, stream);
     if (rc != MS_OK) return rc;
   }
   if (p->d_seg_start) {

@@ -57,8 +57,10 @@ def problem_from_inputs(inp, layer=0, q=None, k_step=None):
                 k_step=inp.k_step if k_step is None else k_step, v_step=inp.v_step, anchor=None)
 
 
-def gpu_attn(P, sm_scale=0.0, want_lse=True, canary=True, device="cuda"):
-    """Runs memosight_attn_step; returns (out bf16 [T][Hq][D] on host, lse fp32 [T][Hq] on host)."""
+def gpu_attn(P, sm_scale=0.0, want_lse=True, canary=True, device="cuda", ws_min_bytes=0):
+    """Runs memosight_attn_step; returns (out bf16 [T][Hq][D] on host, lse fp32 [T][Hq] on host).
+    The workspace has exactly the size the library asks for (or ws_min_bytes if that is more) and
+    a canary region behind it that must come back untouched."""
     dev = torch.device(device)
     d = {k: (v.to(dev) if torch.is_tensor(v) else v) for k, v in P.items()}
     T, Hq, D = P["T"], P["Hq"], P["D"]
@@ -70,7 +72,10 @@ def gpu_attn(P, sm_scale=0.0, want_lse=True, canary=True, device="cuda"):
     max_kv = max(P["lens"] + [0])
     ws_bytes = ms.memosight_attn_workspace_bytes(P["B"], Hq, P["Hkv"], D, max_kv, P["max_nq"])
     assert ws_bytes > 0
-    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    ws_bytes = max(ws_bytes, ws_min_bytes)
+    guard = 1 << 16
+    ws_buf = torch.full((ws_bytes + guard,), 0xA5, dtype=torch.uint8, device=dev)
+    ws = ws_buf[:ws_bytes]
     ms.memosight_attn_step(
         batch=P["B"], n_q_heads=Hq, n_kv_heads=P["Hkv"], head_dim=D, k_cache=d["k_cache"], v_cache=d["v_cache"],
         kv_head_stride=P["n_slots"] * D, n_slots=P["n_slots"], kv_off=d["kv_off"], kv_len=d["kv_len"],
@@ -78,6 +83,7 @@ def gpu_attn(P, sm_scale=0.0, want_lse=True, canary=True, device="cuda"):
         total_rows=T, sm_scale=sm_scale, q=d["q"], k_step=d["k_step"], v_step=d["v_step"], out=out,
         lse=lse if want_lse else None, workspace=ws, workspace_bytes=ws_bytes)
     assert ms.memosight_attn_status(ws) == ms.MS_OK
+    assert bool(torch.all(ws_buf[ws_bytes:] == 0xA5)), "workspace overrun"
     if canary:
         assert torch.all(out_buf[:pad] == 7.0) and torch.all(out_buf[pad + T * Hq * D:] == 7.0), "out overrun"
         if want_lse:

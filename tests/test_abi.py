@@ -51,7 +51,8 @@ def test_host_side_validation_codes():
     assert L.memosight_kv_compact(None, None, 1, 0, 0, 1, 1, 12, None, None, None, None, None, 0, 0, None) \
         == ms.MS_ERR_UNSUPPORTED_SHAPE
     assert L.memosight_kv_compact(None, None, 1, 0, 0, 0, 1, 64, None, None, None, None, None, 0, 0, None) == ms.MS_OK
-    assert L.memosight_kv_append(None, None, 0, 2, 1, 64, None, None, None, None, None, None, None, 4, 1, None) \
+    assert L.memosight_kv_append(None, None, 0, 0, 2, 1, 64, None, None, None, None, None, None, None, None, 4, 1,
+                                 None, None) \
         == ms.MS_ERR_INVALID_ARG
     assert L.memosight_attn_workspace_bytes(1, 5, 2, 64, 10, 4) == 0          # H_q % H_kv != 0
     assert L.memosight_attn_workspace_bytes(1, 4, 2, 64, 10, 32769) == 0        # block too large

@@ -67,7 +67,8 @@ def test_large_block_equals_the_same_tokens_as_small_blocks():
     first = dict(P, T=16, max_nq=16, q=P["q"][:16], k_step=P["k_step"][:16], v_step=P["v_step"][:16],
                  q_off=torch.tensor([0, 16], dtype=torch.int32), n_cand=torch.tensor([16], dtype=torch.int32))
     out1, _ = gpu_attn(first)
-    ms.memosight_kv_append(kc, vc, stride, 1, Hkv, D, P["kv_off"].to(dev), kv_len, P["k_step"][:16].to(dev),
+    ms.memosight_kv_append(kc, vc, stride, P["n_slots"], 1, Hkv, D, P["kv_off"].to(dev), kv_len, None,
+                           P["k_step"][:16].to(dev),
                            P["v_step"][:16].to(dev), first["q_off"].to(dev), first["n_cand"].to(dev),
                            torch.tensor([16], dtype=torch.int32, device=dev), 16, 1)
     torch.cuda.synchronize()

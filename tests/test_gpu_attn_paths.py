@@ -138,3 +138,19 @@ def test_paths_agree_with_each_other(force_path):
     ref = outs["general"].float()
     for path in FAST:
         assert (outs[path].float() - ref).abs().max() <= 2e-2, path
+
+
+@pytest.mark.parametrize("G,nq", [(7, 12), (8, 16), (8, 9)])
+def test_forced_rows_path_never_outgrows_the_workspace(force_path, G, nq):
+    # head_dim 128 with 65..128 packed rows: the automatic choice is the large-block kernel, whose
+    # workspace is small; the rows-on-lanes kernel needs two partial slots per CTA.  Forced with
+    # the workspace the library asks for, the call must fall back (and stay inside the workspace:
+    # the harness checks a canary behind it); forced with a workspace large enough for it, the
+    # rows-on-lanes kernel itself runs.  Both agree with the oracle.
+    lens = [3000, 130, 0, 515]
+    P = random_problem(4, G, 1, 128, lens, [nq, nq - 3, nq, 1], [nq // 2, 2, nq, 1], seed=G * 100 + nq, anchors=True)
+    force_path("tcgen05_rows")
+    check_attn(P, f"forced rows-on-lanes, default workspace G={G} nq={nq}")
+    want, want_lse = oracle_attn(P)
+    out, lse = gpu_attn(P, ws_min_bytes=64 << 20)
+    assert_attn_close(out, lse, want, want_lse, f"forced rows-on-lanes, large workspace G={G} nq={nq}")

@@ -119,8 +119,8 @@ def test_loop_matches_oracle_loop(d, hit, c):
             keep_o = od.commit(seqs, p, q_off_h, am_o, nm_o)
             ms.memosight_decode_commit(st, q_off, am, nm, n_keep)
             for layer, (gks, gvs, k_o, v_o) in enumerate(layers):
-                ms.memosight_kv_append(gk[layer], gv[layer], stride, B, Hkv, D, g_off, g_len, gks, gvs, q_off,
-                                       n_blk, n_keep, 2 * d + 1, layer == NL - 1)
+                ms.memosight_kv_append(gk[layer], gv[layer], stride, n_slots, B, Hkv, D, g_off, g_len, None, gks, gvs,
+                                       q_off, n_blk, n_keep, 2 * d + 1, layer == NL - 1)
                 oracle.kv_append(kb[layer], vb[layer], stride, Hkv, D, kv_off, o_len, k_o, v_o, q_off_h, n_blk_h,
                                  keep_o, bump=(layer == NL - 1))
             torch.cuda.synchronize()
@@ -137,8 +137,8 @@ def test_loop_matches_oracle_loop(d, hit, c):
             q_off_h, n_blk_h, row_tok_h, pos_h, keep_o, seg_s_o, seg_l_o = o_c
             am_o, _, layers = forward(q_off_h, n_blk_h, row_tok_h, pos_h, np.full(T, -1, np.int32), max_mem + 1)
             for layer, (gks, gvs, k_o, v_o) in enumerate(layers):
-                ms.memosight_kv_append(gk[layer], gv[layer], stride, B, Hkv, D, g_off, g_len, gks, gvs, q_off,
-                                       n_blk, n_keep, max_mem + 1, layer == NL - 1)
+                ms.memosight_kv_append(gk[layer], gv[layer], stride, n_slots, B, Hkv, D, g_off, g_len, None, gks, gvs,
+                                       q_off, n_blk, n_keep, max_mem + 1, layer == NL - 1)
                 oracle.kv_append(kb[layer], vb[layer], stride, Hkv, D, kv_off, o_len, k_o, v_o, q_off_h, n_blk_h,
                                  keep_o, bump=(layer == NL - 1))
             ms.memosight_kv_compact(gk, gv, NL, lstride, stride, B, Hkv, D, g_off, g_len, seg_s, seg_l, None, 0,

@@ -68,8 +68,8 @@ def test_captured_step_replays_like_the_eager_step(cfg):
             k_step=t["ks"], v_step=inp.v_step, out=t["out"], lse=t["lse"], workspace=t["ws"], workspace_bytes=wsb)
         ms.memosight_accept(acc.logits, acc.ld_v, cfg.vocab, acc.row_off, B, T, acc.draft, t["am"], t["nm"], t["nk"],
                             t["aws"], awb)
-        ms.memosight_kv_append(inp.k_cache[0], inp.v_cache[0], stride, B, Hkv, D, inp.kv_off, inp.kv_len, t["ks"],
-                               inp.v_step, inp.q_off, inp.n_cand, t["nk"], nq, 1)
+        ms.memosight_kv_append(inp.k_cache[0], inp.v_cache[0], stride, inp.n_slots, B, Hkv, D, inp.kv_off, inp.kv_len,
+                               None, t["ks"], inp.v_step, inp.q_off, inp.n_cand, t["nk"], nq, 1)
         ms.memosight_kv_compact(inp.k_cache, inp.v_cache, 1, Hkv * stride, stride, B, Hkv, D, inp.kv_off,
                                 inp.kv_len, seg_start, seg_len, None, 0, 5)
 

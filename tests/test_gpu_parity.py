@@ -198,7 +198,7 @@ def test_append_accepted_candidates():
     oracle.kv_append(kb, vb, inp.n_slots * 128, 2, 128, inp.kv_off.numpy(), kv_len, bits(inp.k_step),
                      bits(inp.v_step), inp.q_off.numpy(), inp.n_cand.numpy(), [0, 1, 4, 2, 4])
     gk, gv, g_len = inp.k_cache[0].to(DEV).clone(), inp.v_cache[0].to(DEV).clone(), inp.kv_len.to(DEV).clone()
-    args = (gk, gv, inp.n_slots * 128, 5, 2, 128, inp.kv_off.to(DEV), g_len, inp.k_step.to(DEV),
+    args = (gk, gv, inp.n_slots * 128, inp.n_slots, 5, 2, 128, inp.kv_off.to(DEV), g_len, None, inp.k_step.to(DEV),
             inp.v_step.to(DEV), inp.q_off.to(DEV), inp.n_cand.to(DEV),
             torch.tensor(n_keep, dtype=torch.int32, device=DEV), cfg.n_q)
     ms.memosight_kv_append(*args, 0)
@@ -208,6 +208,49 @@ def test_append_accepted_candidates():
     torch.cuda.synchronize()
     assert np.array_equal(g_len.cpu().numpy(), kv_len)
     assert np.array_equal(bits(gk), kb) and np.array_equal(bits(gv), vb)   # whole buffers, untouched slots too
+
+
+@pytest.mark.parametrize("with_cap", [True, False])
+def test_append_stops_at_the_capacity(with_cap):
+    # Sequences that have (almost) no room left: the append takes what fits, reports it, moves the
+    # length by that much, and writes neither into the neighbour's slots nor behind the tensor.
+    cfg = synth.StepConfig("cap", 3, 8, 2, 128, 30, 90, 4, 2, 1e4, 100, headroom=2, seed=80)
+    inp = synth.make_step_inputs(cfg)
+    n_slots, D, Hkv = inp.n_slots, 128, 2
+    if with_cap:
+        want_keep = [4, 2, 4]
+        cap = [inp.lens[0] + 1, inp.lens[1] + 2, inp.lens[2]]            # room for 1, for 2, for none
+        room = [1, 2, 0]
+    else:
+        want_keep = [2, 2, 4]
+        cap = None
+        room = [2, 2, 2]            # every sequence has 2 free slots; behind the last one the tensor ends
+    keep = [min(w, r) for w, r in zip(want_keep, room)]
+    kb, vb = bits(inp.k_cache[0]), bits(inp.v_cache[0])
+    kv_len = inp.kv_len.numpy().copy()
+    oracle.kv_append(kb, vb, n_slots * D, Hkv, D, inp.kv_off.numpy(), kv_len, bits(inp.k_step), bits(inp.v_step),
+                     inp.q_off.numpy(), inp.n_cand.numpy(), keep)
+    # the cache tensors sit inside larger buffers whose surroundings must not change
+    guard = 4096
+    def guarded(t):
+        buf = torch.full((t.numel() + 2 * guard,), 7.0, dtype=torch.bfloat16, device=DEV)
+        view = buf[guard:guard + t.numel()].view(t.shape)
+        view.copy_(t)
+        return buf, view
+    kbuf, gk = guarded(inp.k_cache[0])
+    vbuf, gv = guarded(inp.v_cache[0])
+    g_len = inp.kv_len.to(DEV).clone()
+    flag = torch.zeros(1, dtype=torch.int32, device=DEV)
+    ms.memosight_kv_append(gk, gv, n_slots * D, n_slots, 3, Hkv, D, inp.kv_off.to(DEV), g_len,
+                           None if cap is None else torch.tensor(cap, dtype=torch.int32, device=DEV),
+                           inp.k_step.to(DEV), inp.v_step.to(DEV), inp.q_off.to(DEV), inp.n_cand.to(DEV),
+                           torch.tensor(want_keep, dtype=torch.int32, device=DEV), cfg.n_q, 1, flag)
+    torch.cuda.synchronize()
+    assert g_len.tolist() == [L + k for L, k in zip(inp.lens, keep)]
+    assert int(flag.item()) == 1
+    assert np.array_equal(bits(gk), kb) and np.array_equal(bits(gv), vb)
+    for buf in (kbuf, vbuf):
+        assert bool(torch.all(buf[:guard] == 7.0)) and bool(torch.all(buf[-guard:] == 7.0)), "wrote outside the tensor"
 
 
 # --------------------------------------------------------------------------- accept
@@ -238,6 +281,14 @@ def test_accept_tiny_and_planted_prefix_lengths():
         am, nm = _accept_both(a.logits, cfg.vocab, a.row_off.tolist(), a.draft.tolist())
         assert am.tolist() == a.target
     assert set(nm.tolist()) == set(range(5))          # every prefix length 0..n_c-1 occurs
+
+
+def test_accept_many_sequences_takes_the_two_launch_form():
+    # more rows than the in-kernel tail has counters for: pass 2 is then a launch of its own
+    cfg = synth.StepConfig("acc-wide", 700, 4, 2, 64, 8, 8, 2, 1, 1e4, 8192 + 64, seed=15)
+    a = synth.make_accept_inputs(cfg)
+    am, nm = _accept_both(a.logits, cfg.vocab, a.row_off.tolist(), a.draft.tolist())
+    assert am.tolist() == a.target and set(nm.tolist()) == {0, 1}
 
 
 def test_accept_unplanted_ties_nan_inf_and_unaligned_rows():
@@ -335,7 +386,7 @@ def test_whole_step_chain_rope_attn_accept_append():
     ms.memosight_accept(acc.logits.to(DEV), acc.ld_v, cfg.vocab, acc.row_off.to(DEV), B, T, acc.draft.to(DEV),
                         am, nm, nk, ws, wsb)
     gk, gv, g_len = inp.k_cache[0].to(DEV).clone(), inp.v_cache[0].to(DEV).clone(), inp.kv_len.to(DEV).clone()
-    ms.memosight_kv_append(gk, gv, inp.n_slots * 128, B, 2, 128, inp.kv_off.to(DEV), g_len, ks, vs,
+    ms.memosight_kv_append(gk, gv, inp.n_slots * 128, inp.n_slots, B, 2, 128, inp.kv_off.to(DEV), g_len, None, ks, vs,
                            inp.q_off.to(DEV), inp.n_cand.to(DEV), nk, nq, 1)
     torch.cuda.synchronize()
     assert np.array_equal(am.cpu().numpy(), am_o) and np.array_equal(nm.cpu().numpy(), nm_o)

@@ -58,8 +58,8 @@ def test_step_host_equals_the_separate_calls_two_steps():
             v_step=inp.v_step, out=t["out"], lse=None, workspace=t["ws"], workspace_bytes=wsb)
         a = accs[s]
         ms.memosight_accept(a.logits, a.ld_v, cfg.vocab, a.row_off, B, T, a.draft, t["am"], t["nm"], t["nk"], t["aws"], awb)
-        ms.memosight_kv_append(inp.k_cache[0], inp.v_cache[0], stride, B, Hkv, D, inp.kv_off, inp.kv_len, ks,
-                               inp.v_step, inp.q_off, inp.n_cand, t["nk"], nq, 1)
+        ms.memosight_kv_append(inp.k_cache[0], inp.v_cache[0], stride, inp.n_slots, B, Hkv, D, inp.kv_off, inp.kv_len,
+                               None, ks, inp.v_step, inp.q_off, inp.n_cand, t["nk"], nq, 1)
         if s == 0:
             ms.memosight_kv_compact(inp.k_cache, inp.v_cache, 1, Hkv * stride, stride, B, Hkv, D, inp.kv_off,
                                     inp.kv_len, seg_start, seg_len, None, 0, 20)

@@ -3,12 +3,14 @@ memory (a frozen serving allocator, a plug-in without an allocator handle).  Its
 scratch is a fixed array inside the library, shared by every call and never cleared,
 so the check is made on two calls in a row with different inputs: both must equal what
 memosight_accept (caller workspace) returns, bit for bit -- stale contents of the shared
-array must not matter.  Collected last on purpose: a failure here cannot hide another
-test's result in a run that stops at the first failure."""
+array must not matter -- and what the CPU oracle's accept returns for the same logits, so that
+a mistake the two launch paths had in common would not pass either.  Collected last on purpose:
+a failure here cannot hide another test's result in a run that stops at the first failure."""
 import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2604_14889_b200 import binding as ms
 from paper_2604_14889_b200 import synth
 
@@ -27,6 +29,10 @@ def _both(cfg, plant, pad):
     torch.cuda.synchronize()
     for g, r in zip(got, ref):
         assert torch.equal(g, r)
+    want_am, want_nm = oracle.accept(a.logits.cpu().numpy(), cfg.vocab, a.row_off.cpu().numpy(), a.draft.cpu().numpy())
+    assert np.array_equal(got[0].cpu().numpy(), want_am)
+    assert np.array_equal(got[1].cpu().numpy(), want_nm)
+    assert np.array_equal(got[2].cpu().numpy(), want_nm + 1)
     return a, got
 
 
