@@ -40,12 +40,13 @@ from paper_2604_14889_b200 import synth
 
 METRIC = "step query tokens/s (Predict+Verify attention step, 8B-shape, compacted KV 16K)"
 UNIT = "tokens/s"
+METRIC_CONFIG = "step query tokens/s (Predict+Verify step of the named configuration: RoPE, attention, accept, append, all layers)"
 SEG_LEN, MEM_TOKENS = 512, 170          # one compaction: 512-token step -> 170 memory tokens + <o>
 FALLBACK_HBM_GBS = 6650.0
-# DRAM bytes the split kernel moved per algorithmic byte in the ncu capture summarised in
-# profiles/attn_umma_t_kernel_sweep_b32_L16384.md (batch 32; scaled by the bytes streamed).
+# DRAM bytes the split kernel moved per algorithmic byte in an ncu capture of the batch-32 point
+# of the same workload (scaled by the bytes streamed).
 NCU_TRAFFIC_PER_ALGO_BYTE = 1.011
-KERNELS_PER_STEP = 9                    # rope 1, attention 2, accept 2, append 2, compaction 2
+KERNELS_PER_STEP = 5                    # rope, attention (merge in its tail), accept, append, compaction
 
 
 def parse_args():
@@ -61,9 +62,11 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample-seqs", type=int, default=32)
-    ap.add_argument("--workload", default="step", choices=["step", "compress"],
+    ap.add_argument("--workload", default="step", choices=["step", "compress", "loop", "cacheops"],
                     help="step: the Predict+Verify step the headline metric is quoted on (default); "
-                         "compress: the compression event (forward of the memory tokens + <o>, append, eviction)")
+                         "compress: the compression event (forward of the memory tokens + <o>, append, eviction); "
+                         "loop: the whole inference loop of Algorithm 1 with a toy model, d = 0..4 x c = 3, 5 x batch 1, 64; "
+                         "cacheops: compaction, keep-list eviction, RoPE, append and merge kernels, each timed alone")
     ap.add_argument("--sweep", action="store_true",
                     help="the foresight/batch/cache-length sweep (8B shape): one device-resident run per point, "
                          "a table of KV bytes read, step tokens/s and HBM fraction on stdout")
@@ -73,6 +76,12 @@ def parse_args():
     ap.add_argument("--uncompressed", action="store_true",
                     help="the cache is an uncompressed one (position IDs = cache indices); with --kv-len 49152 "
                          "it is the counterpart of the compacted 16K cache")
+    ap.add_argument("--config", default=None, choices=["tiny", "qwen7b", "llama8b-ragged", "longcot", "all"],
+                    help="one of the named workload configurations (ragged lengths, its own shapes and vocabulary) "
+                         "instead of the headline sweep point; 'all' runs the four one after the other (a process "
+                         "each) and prints a table")
+    ap.add_argument("--layers", type=int, default=0, help="--config longcot: logical layers (default 32)")
+    ap.add_argument("--cpu-only", action="store_true", help=argparse.SUPPRESS)
     ap.add_argument("--attn-path", default="auto", choices=["auto", "mma_sync", "tcgen05", "tcgen05_keys"],
                     help="attention kernel: by shape (default), or forced for A/B timing")
     return ap.parse_args()
@@ -261,7 +270,8 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": workload_config(cfg, args),
+        "config": dict(workload_config(cfg, args), sample="each timed step is one whole hot-path step of ONE of the "
+                                                          "workload's sequences (the oracle is far too slow for the batch)"),
         "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle",
                          "sample": "each step = one whole hot-path step of 1 of the workload's sequences"},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -304,9 +314,10 @@ def run_sweep(args):
     prints one table row per point plus the JSON lines."""
     import subprocess
     rows, lines = [], []
-    print("| d | batch | cache | KV GB/step | step ms | step ms (CUDA graph) | attention µs | step tokens/s | "
-          "step tokens/s (CUDA graph) | attention GB/s | of measured HBM | of 8 TB/s |")
-    print("|---:|---:|---|---:|---:|---:|---:|---:|---:|---:|---:|---:|", flush=True)
+    print("| d | batch | cache | KV GB/step | step ms (5 Python calls) | step ms (one call) | step ms (CUDA graph) | "
+          "attention µs | step tokens/s (one call) | step tokens/s (CUDA graph) | attention GB/s | of measured HBM | "
+          "of 8 TB/s |")
+    print("|---:|---:|---|---:|---:|---:|---:|---:|---:|---:|---:|---:|---:|", flush=True)
     for kv_len, unc in ((16384, False), (49152, True)):
         for d in range(1, 8):
             for batch in (1, 8, 32, 128):
@@ -321,8 +332,9 @@ def run_sweep(args):
                 lines.append(j)
                 r = j["roofline"]
                 print(f"| {d} | {batch} | {'48K uncompressed' if unc else '16K compacted'} | {j['kv_gb_per_step']:.3f} | "
-                      f"{j['ms_per_step']:.3f} | {j['graph']['ms_per_step']:.3f} | {r['avg_launch_ms'] * 1e3:.1f} | "
-                      f"{j['value']:.0f} | {j['graph']['value']:.0f} | {r['achieved']:.0f} | "
+                      f"{j['ms_per_step']:.3f} | {j['one_call']['ms_per_step']:.3f} | {j['graph']['ms_per_step']:.3f} | "
+                      f"{r['avg_launch_ms'] * 1e3:.1f} | {j['one_call']['value']:.0f} | {j['graph']['value']:.0f} | "
+                      f"{r['achieved']:.0f} | "
                       f"{r['frac']:.2f}{' (L2)' if j['kv_gb_per_step'] < 0.5 else ''} | {r['frac_of_nominal_8000']:.2f} |",
                       flush=True)
     for j in lines:
@@ -336,6 +348,12 @@ def main():
         return
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.config == "all":
+        run_all_configs(args)
+        return
+    if args.config and args.cpu_only:
+        print(json.dumps(config_cpu_baseline(CONFIGS[args.config](), args.config)), flush=True)
         return
     from paper_2604_14889_b200 import binding as ms
 
@@ -355,13 +373,23 @@ def main():
     if args.workload == "compress":
         run_compress(args, ms, dev, world, rank)
         return
+    if args.workload == "loop":
+        run_loop(args, ms, dev)
+        return
+    if args.workload == "cacheops":
+        run_cacheops(args, ms, dev)
+        return
+    if args.config:
+        assert world == 1, "--config is a single-GPU measurement"
+        run_config(args, ms, dev)
+        return
     K, W = args.steps, max(args.warmup, 3)
     cfg0 = synth.sweep(args.batch, args.d, args.kv_len, not args.uncompressed)
     n_e2e = 0 if args.no_e2e else max(1, min(args.e2e_steps, K))
     n_total = W + K
     if args.graph and n_e2e:
         raise SystemExit("--graph needs --no-e2e")
-    n_sched = n_total + (3 + n_e2e if n_e2e else 0) + (K + 1 if args.graph else 0)
+    n_sched = n_total + (3 + n_e2e if n_e2e else 0) + (2 * K + 1 if args.graph else 0)
     growth = 3 * n_sched + SEG_LEN + 64
     cfg = synth.StepConfig(cfg0.name, cfg0.batch, cfg0.n_q_heads, cfg0.n_kv_heads, cfg0.head_dim, cfg0.len_lo,
                            cfg0.len_hi, cfg0.n_cand, cfg0.d, cfg0.rope_base, cfg0.vocab, headroom=growth,
@@ -464,6 +492,39 @@ def main():
         graph_info = {"ms_per_step": g_ms / K, "value": g_value, "unit": UNIT,
                       "note": "K further steps captured once in a CUDA graph, one replay timed"}
 
+    one_call = None
+    if args.graph:
+        # the same step queued by ONE call into the library (memosight_step_host with no host buffers):
+        # what an eager step costs a caller that does not go through five Python calls
+        import ctypes as C
+        sp = ms.StepHostParams()
+        sp.struct_size = C.sizeof(ms.StepHostParams)
+        sp.attn = plain
+        sp.d_pos_id = pos.data_ptr()
+        sp.rope_base, sp.rope_flags, sp.vocab = cfg.rope_base, 0, cfg.vocab
+        sp.ld_v, sp.d_logits, sp.d_draft = acc.ld_v, acc.logits.data_ptr(), acc.draft.data_ptr()
+        sp.d_argmax, sp.d_n_match, sp.d_n_keep = am.data_ptr(), nm.data_ptr(), nk.data_ptr()
+        sp.accept_workspace, sp.accept_workspace_bytes = aws.data_ptr(), awb
+        sp.max_tail = MEM_TOKENS + 1
+        first = n_total + K
+        o0, o1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+        def call_step(s):
+            sp.d_seg_start, sp.d_seg_len = seg_start[s].data_ptr(), seg_len[s].data_ptr()
+            ms.memosight_step_host(sp)
+        call_step(first)
+        barrier()
+        o0.record()
+        for s in range(K):
+            call_step(first + 1 + s)
+        o1.record()
+        barrier()
+        assert ms.memosight_attn_status(ws) == ms.MS_OK
+        assert inp.kv_len.cpu().tolist() == sched.final, "one-call steps: cache lengths differ"
+        oc_value, oc_ms = whole_job_throughput(T * K, o0.elapsed_time(o1), world, dev)
+        one_call = {"ms_per_step": oc_ms / K, "value": oc_value, "unit": UNIT,
+                    "note": "K further eager steps, each queued by one memosight_step_host call without host buffers"}
+
     # roofline of the dominant kernel (split-KV attention): algorithmic KV bytes per launch / its duration
     kv_bytes = [sched.kv_bytes(W + s, cfg) for s in range(K)]
     step_local = T * (2 * Hq + 2 * Hkv) * D * 2
@@ -486,12 +547,14 @@ def main():
 
     # ---- end to end: the step's inputs and results live in pinned host memory
     e2e = None
-    if not args.no_e2e and rank == 0:
+    if not args.no_e2e:
+        # every rank runs its own end-to-end steps; the job's time is the slowest rank's
         e2e = run_e2e(ms, n_e2e, n_total, cfg, inp, acc, sched, seg_start, seg_len, ws, wsb, aws, awb, am, nm,
                       nk, out, lse, pos, max_kv)
-    if world > 1 and e2e is not None:
-        e2e["note"] = "measured on rank 0 only, scaled by the number of ranks"
-        e2e["value"] *= world
+        e2e["value"], e2e_ms = whole_job_throughput(T * n_e2e, e2e["ms_per_step"] * n_e2e, world, dev)
+        e2e["ms_per_step"] = e2e_ms / n_e2e
+        if world > 1:
+            e2e["note"] = "every rank measured; time = max over ranks, tokens = sum over ranks"
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
@@ -505,6 +568,8 @@ def main():
         line["e2e"] = e2e
     if graph_info is not None:
         line["graph"] = graph_info
+    if one_call is not None:
+        line["one_call"] = one_call
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
             del inp, acc
@@ -515,6 +580,835 @@ def main():
         import torch.distributed as dist
         dist.barrier()
         dist.destroy_process_group()
+
+
+
+# --------------------------------------------------------------------------- the named configurations
+
+CONFIGS = {"tiny": lambda: synth.TINY, "qwen7b": lambda: synth.QWEN7B,
+           "llama8b-ragged": lambda: synth.LLAMA8B_RAGGED, "longcot": lambda: synth.LONGCOT}
+COLD_BYTES = 512e6            # small caches rotate over copies worth at least this much, so that reads come from HBM
+
+
+def config_cpu_baseline(cfg, name, min_seconds=4.0):
+    """The oracle, as it stands, on the host cores: whole steps (one layer) of the configuration --
+    every sequence for the first three, a seeded subset extrapolated linearly for the long-CoT one."""
+    import oracle
+    full = name != "longcot"
+    n_seqs = cfg.batch if full else 4
+    sub = synth.StepConfig(cfg.name + "-cpu", n_seqs, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.len_lo,
+                           cfg.len_hi, cfg.n_cand, cfg.d, cfg.rope_base, cfg.vocab, headroom=64, seed=cfg.seed)
+    lens = synth.make_lengths(cfg)[:n_seqs]
+    inp = synth.make_step_inputs(sub, lens=lens)
+    acc = synth.make_accept_inputs(sub)
+    D, Hkv = sub.head_dim, sub.n_kv_heads
+    kb, vb = bits(inp.k_cache), bits(inp.v_cache)
+    qb, ksb, vsb = bits(inp.q), bits(inp.k_step), bits(inp.v_step)
+    stride = inp.n_slots * D
+
+    def step():
+        pid = np.concatenate([oracle.step_pids(inp.p0[b], sub.n_cand, sub.d) for b in range(n_seqs)])
+        q_r, k_r = oracle.rope(qb, pid, sub.rope_base), oracle.rope(ksb, pid, sub.rope_base)
+        lens_now = inp.kv_len.numpy().copy()
+        oracle.attn_step(kb[0], vb[0], stride, inp.kv_off.numpy(), lens_now, inp.q_off.numpy(), inp.n_cand.numpy(),
+                         None, q_r, k_r, vsb)
+        _, nm = oracle.accept(acc.logits.numpy(), sub.vocab, acc.row_off.numpy(), acc.draft.numpy())
+        oracle.kv_append(kb[0], vb[0], stride, Hkv, D, inp.kv_off.numpy(), lens_now, k_r, vsb, inp.q_off.numpy(),
+                         inp.n_cand.numpy(), nm + 1)
+
+    step()
+    n, t0 = 0, time.perf_counter()
+    while n == 0 or (time.perf_counter() - t0 < min_seconds and n < 200):
+        step()
+        n += 1
+    dt = (time.perf_counter() - t0) / n
+    kv_bytes = sum(lens) * Hkv * D * 4
+    scale = 1.0 if full else cfg.batch / n_seqs
+    layers = 1 if full else 32
+    out = {"value": cfg.batch * sub.n_q / (dt * scale * layers), "unit": UNIT, "cores": oracle.threads(),
+           "kind": "oracle", "ms_per_layer_step": dt * 1e3 * scale, "effective_gbs": kv_bytes / dt / 1e9,
+           "sample": (f"{n} whole one-layer steps (rope, attention, accept, append) of all {n_seqs} sequences"
+                      if full else
+                      f"{n} whole one-layer steps of {n_seqs} of the {cfg.batch} sequences; ms_per_layer_step is "
+                      f"extrapolated linearly to the batch (x{scale:.0f}), value to 32 layers -- extrapolated")}
+    return out
+
+
+def run_all_configs(args):
+    import subprocess
+    lines = []
+    for name in ("tiny", "qwen7b", "llama8b-ragged", "longcot"):
+        cmd = [sys.executable, os.path.abspath(__file__), "--config", name, "--steps", str(args.steps), "--warmup",
+               str(args.warmup)] + (["--no-cpu-baseline"] if args.no_cpu_baseline else [])
+        out = subprocess.run(cmd, capture_output=True, text=True)
+        if out.returncode != 0:
+            print(out.stderr[-3000:], file=sys.stderr)
+            raise SystemExit(out.returncode)
+        lines.append(json.loads(out.stdout.strip().splitlines()[-1]))
+    print("| config | batch | layers | rows | KV GB/step | step ms | step ms (CUDA graph) | step tokens/s (CUDA graph) | attention ms/step | attention GB/s | "
+          "of measured HBM | of 8 TB/s | L2-warm attention GB/s | rope µs | accept µs | append µs | compaction event µs "
+          "(amortised µs/step) | oracle tokens/s (cores) |")
+    print("|---|---:|---:|---:|---:|---:|---:|---:|---:|---:|---:|---:|---:|---:|---:|---:|---:|---:|")
+    for j in lines:
+        r, c, pt = j["roofline"], j["config"], j["parts"]
+        cb = j.get("cpu_baseline")
+        warm = j.get("l2_warm")
+        print(f"| {c['name']} | {c['global_batch']} | {c['layers']} | {c['rows']} | {j['kv_gb_per_step']:.4f} | "
+              f"{j['ms_per_step']:.4f} | {j['graph']['ms_per_step']:.4f} | {j['graph']['value']:.0f} | "
+              f"{r['avg_launch_ms'] * r['launches_per_step']:.4f} | "
+              f"{r['achieved']:.0f} | {r['frac']:.2f} | {r['frac_of_nominal_8000']:.2f} | "
+              f"{'' if warm is None else format(warm['achieved'], '.0f')} | {pt['rope_us']:.1f} | {pt['accept_us']:.1f} | "
+              f"{pt['append_us']:.1f} | {pt['compaction_event_us']:.1f} ({pt['compaction_amortised_us_per_step']:.2f}) | "
+              f"{'' if cb is None else format(cb['value'], '.1f') + ' (' + str(cb['cores']) + ')'} |")
+    for j in lines:
+        print(json.dumps(j))
+
+
+def run_config(args, ms, dev):
+    """One named configuration, device-resident.  A step = for every layer: RoPE of the block at its
+    position IDs -> step attention -> append of the accepted candidates; once per step the greedy
+    accept.  The long-CoT configuration stacks 32 logical layers over as many physical cache layers
+    as fit in 70 % of the free memory (each layer is far larger than the L2, so cycling over them
+    reuses nothing), issues its attention through the stacked-layer entry (and, for comparison, layer
+    by layer) and times its compaction event (every sequence, every layer, 512 -> 170 + <o>)
+    separately: the event happens once per 512 generated tokens and is reported amortised.  The two
+    small configurations rotate over enough copies of their cache to exceed 512 MB, so that their
+    bandwidth is an HBM figure; the figure with one copy (L2-warm) is reported beside it."""
+    name = args.config
+    cfg0 = CONFIGS[name]()
+    K, W = args.steps if args.steps != 200 else 50, max(args.warmup, 3)
+    B, Hq, Hkv, D, nq = cfg0.batch, cfg0.n_q_heads, cfg0.n_kv_heads, cfg0.head_dim, cfg0.n_q
+    T = B * nq
+    lens0 = synth.make_lengths(cfg0)
+    n_rounds = 4                                    # whole, graph, parts, per-layer (or L2-warm)
+    growth = cfg0.n_cand * (W + K + 2) * (n_rounds + 1) + 64
+    if name == "longcot":
+        growth = max(growth, SEG_LEN + MEM_TOKENS + 64)
+    layer_bytes = 2 * Hkv * (sum(lens0) + B * growth) * D * 2
+    NL = (args.layers or 32) if name == "longcot" else 1
+    if name == "longcot":
+        free, _ = torch.cuda.mem_get_info()
+        n_phys = max(1, min(NL, int(0.7 * free // layer_bytes)))
+    elif layer_bytes < COLD_BYTES:
+        n_phys = int(-(-COLD_BYTES // layer_bytes))
+    else:
+        n_phys = 1
+    cfg = synth.StepConfig(cfg0.name, B, Hq, Hkv, D, cfg0.len_lo, cfg0.len_hi, cfg0.n_cand, cfg0.d, cfg0.rope_base,
+                           cfg0.vocab, n_layers=n_phys, headroom=growth, seed=cfg0.seed)
+    inp = synth.make_step_inputs(cfg, device=dev, lens=lens0)
+    acc = synth.make_accept_inputs(cfg, device=dev)
+    keep = [synth.hash_scalar(b, cfg.seed, synth.STREAM_ACCEPT) % max(cfg.n_cand, 1) + 1 for b in range(B)]
+    stride, lstride = inp.n_slots * D, Hkv * inp.n_slots * D
+    max_kv = max(lens0) + growth
+    pos1 = np.concatenate([ms.memosight_step_pids(inp.p0[b], cfg.n_cand, cfg.d) for b in range(B)])
+    pos = torch.from_numpy(np.tile(pos1, NL)).to(dev)
+    # step tensors of every logical layer (the same values in every layer: the generator's draw of one layer)
+    q_all = inp.q.unsqueeze(0).repeat(NL, 1, 1, 1).contiguous()
+    ks_all = inp.k_step.unsqueeze(0).repeat(NL, 1, 1, 1).contiguous()
+    vs_all = inp.v_step.unsqueeze(0).repeat(NL, 1, 1, 1).contiguous()
+    out_all = torch.empty((NL, T, Hq, D), dtype=torch.bfloat16, device=dev)
+    wsb = ms.memosight_attn_workspace_bytes(B, Hq, Hkv, D, max_kv, nq)
+    ws = torch.empty(wsb, dtype=torch.uint8, device=dev)
+    awb = ms.memosight_accept_workspace_bytes(T, cfg.vocab)
+    aws = torch.empty(awb, dtype=torch.uint8, device=dev)
+    am = torch.empty(T, dtype=torch.int32, device=dev)
+    nm = torch.empty(B, dtype=torch.int32, device=dev)
+    nk = torch.empty(B, dtype=torch.int32, device=dev)
+    q_ls, ks_ls = T * Hq * D, T * Hkv * D
+    state = {"step": 0}
+
+    def params(phys, logical):
+        return ms.attn_params(
+            batch=B, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, k_cache=inp.k_cache[phys], v_cache=inp.v_cache[phys],
+            kv_head_stride=stride, n_slots=inp.n_slots, kv_off=inp.kv_off, kv_len=inp.kv_len, max_kv_len=max_kv,
+            max_nq=nq, q_off=inp.q_off, n_cand=inp.n_cand, anchor=None, total_rows=T, sm_scale=0.0, q=q_all[logical],
+            k_step=ks_all[logical], v_step=vs_all[logical], out=out_all[logical], lse=None, workspace=ws,
+            workspace_bytes=wsb)
+
+    # stacked issue: runs of consecutive physical layers, the logical layers cycling over them
+    runs = []
+    l = 0
+    while l < NL:
+        n = min(n_phys, NL - l)
+        runs.append((l, n))
+        l += n
+    run_params = [params(0, l0) for l0, _ in runs]
+    layer_params = {}
+
+    def attn(stacked, ev=None, rotate=True):
+        """The attention of one step: all logical layers."""
+        if NL == 1:
+            phys = (state["step"] % n_phys) if rotate else 0
+            key = ("one", phys)
+            if key not in layer_params:
+                layer_params[key] = params(phys, 0)
+            if ev:
+                ms.memosight_attn_debug_events(ev[0].cuda_event, ev[1].cuda_event)
+            ms.memosight_attn_step(layer_params[key])
+            if ev:
+                ms.memosight_attn_debug_events(None, None)
+            return 1
+        n_launch = 0
+        if stacked:
+            for i, (l0, n) in enumerate(runs):
+                if ev:
+                    ms.memosight_attn_debug_events(ev[i][0].cuda_event, ev[i][1].cuda_event)
+                ms.memosight_attn_step_layers(run_params[i], n, lstride, q_ls, ks_ls, q_ls)
+                n_launch += 1
+        else:
+            for lg in range(NL):
+                key = ("layer", lg)
+                if key not in layer_params:
+                    layer_params[key] = params(lg % n_phys, lg)
+                if ev:
+                    ms.memosight_attn_debug_events(ev[lg][0].cuda_event, ev[lg][1].cuda_event)
+                ms.memosight_attn_step(layer_params[key])
+                n_launch += 1
+        if ev:
+            ms.memosight_attn_debug_events(None, None)
+        return n_launch
+
+    def rope():
+        ms.memosight_rope_qk(q_all, ks_all, pos, NL * T, Hq, Hkv, D, cfg.rope_base)
+
+    def accept():
+        ms.memosight_accept(acc.logits, acc.ld_v, cfg.vocab, acc.row_off, B, T, acc.draft, am, nm, nk, aws, awb)
+
+    def append(rotate=True):
+        if NL == 1:
+            phys = (state["step"] % n_phys) if rotate else 0
+            ms.memosight_kv_append(inp.k_cache[phys], inp.v_cache[phys], stride, inp.n_slots, B, Hkv, D, inp.kv_off,
+                                   inp.kv_len, None, ks_all[0], vs_all[0], inp.q_off, inp.n_cand, nk, nq, 1)
+            return
+        for lg in range(NL):
+            # (layers that share a physical cache layer append to the same slots: the bytes moved are what counts)
+            ms.memosight_kv_append(inp.k_cache[lg % n_phys], inp.v_cache[lg % n_phys], stride, inp.n_slots, B, Hkv, D,
+                                   inp.kv_off, inp.kv_len, None, ks_all[lg], vs_all[lg], inp.q_off, inp.n_cand, nk, nq,
+                                   1 if lg == NL - 1 else 0)
+
+    def step(stacked=True, rotate=True):
+        rope()
+        attn(stacked, rotate=rotate)
+        accept()
+        append(rotate)
+        state["step"] += 1
+
+    def timed(fn, n):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        t_host = time.perf_counter()
+        e0.record()
+        for _ in range(n):
+            fn()
+        e1.record()
+        host_ms = (time.perf_counter() - t_host) * 1e3
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n, host_ms / n
+
+    lens_now = list(lens0)
+
+    def advance(n):
+        for b in range(B):
+            lens_now[b] += keep[b] * n
+
+    def kv_bytes_mean(n):
+        """Algorithmic K/V bytes per step (all layers), averaged over the next n steps."""
+        tot = 0
+        for s in range(n):
+            tot += sum(L + keep[b] * s for b, L in enumerate(lens_now))
+        return tot / n * Hkv * D * 4 * NL
+
+    for _ in range(W):
+        step()
+    advance(W)
+    assert ms.memosight_attn_status(ws) == ms.MS_OK
+    sampler = ClockSampler(physical_gpu_index(int(os.environ.get("LOCAL_RANK", "0"))))
+    sampler.start()
+    # ---- round 1: whole steps
+    kv_whole = kv_bytes_mean(K)
+    step_ms, host_ms = timed(step, K)
+    advance(K)
+    clocks = sampler.finish()
+    assert inp.kv_len.cpu().tolist() == lens_now, "cache lengths differ from the replayed schedule"
+    assert nm.cpu().tolist() == [k - 1 for k in keep]
+    # ---- the same K steps captured once in a CUDA graph, one replay timed (what the kernels cost when
+    #      the host's launch work is gone; small configurations are bound by it otherwise)
+    side = torch.cuda.Stream()
+    gr = torch.cuda.CUDAGraph()
+    torch.cuda.synchronize()
+    with torch.cuda.graph(gr, stream=side):
+        for _ in range(K):
+            step()
+    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    g0.record()
+    gr.replay()
+    g1.record()
+    torch.cuda.synchronize()
+    advance(K)
+    assert inp.kv_len.cpu().tolist() == lens_now, "graph replay: cache lengths differ"
+    graph_ms = g0.elapsed_time(g1) / K
+    del gr
+    # ---- round 2: the parts, each bracketed by events (this serialises the launches a little)
+    n_ev = len(runs) if NL > 1 else 1
+    evs = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_ev)]
+           for _ in range(K)]
+    marks = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(K)]
+    for row in evs:
+        for a_, b_ in row:
+            a_.record()
+            b_.record()
+    kv_parts = kv_bytes_mean(K)
+    for s_ in range(K):
+        m = marks[s_]
+        m[0].record()
+        rope()
+        m[1].record()
+        attn(True, ev=evs[s_] if NL > 1 else evs[s_][0])
+        m[2].record()
+        accept()
+        m[3].record()
+        append()
+        m[4].record()
+        state["step"] += 1
+    torch.cuda.synchronize()
+    advance(K)
+    assert ms.memosight_attn_status(ws) == ms.MS_OK
+    part = lambda i: float(np.mean([m[i].elapsed_time(m[i + 1]) for m in marks])) * 1e3
+    split_ms = [sum(a_.elapsed_time(b_) for a_, b_ in row) for row in evs]        # per step, all launches
+    attn_ms = float(np.mean(split_ms))
+    step_local = T * (2 * Hq + 2 * Hkv) * D * 2 * NL
+    algo = kv_parts + step_local
+    achieved = algo / (attn_ms * 1e-3) / 1e9
+    peak, peak_kind = peak_hbm()
+    rows = nq * (Hq // Hkv)
+    if D == 128 and rows <= 64:
+        kernel = f"attn_umma_t_kernel<{(rows + 15) // 16 * 16}>"
+    elif D == 64:
+        kernel = f"attn_split_kernel<64,{1 if rows <= 16 else 2 if rows <= 32 else 4}>"
+    else:
+        kernel = "attn_umma_big_kernel"
+    cold = n_phys > 1 or layer_bytes > 4 * 126e6
+    roofline = {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak,
+                "peak_source": f"{peak_kind} copy bandwidth", "unit": "GB/s", "frac": achieved / peak,
+                "frac_of_nominal_8000": achieved / 8000.0, "avg_launch_ms": attn_ms / n_ev, "launches_per_step": n_ev,
+                "algorithmic_bytes_per_launch": algo / n_ev, "traffic": None,
+                "share_of_step_time": attn_ms / (part(0) + part(1) + part(2) + part(3)) * 1e3,
+                "reads_from": "HBM" if cold else "L2 (the cache is not much larger than the 126 MB L2)"}
+    # ---- round 3: layer by layer (long-CoT) or L2-warm (one copy of a small cache)
+    per_layer, l2_warm = None, None
+    if NL > 1:
+        ev_l = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(NL)]
+                for _ in range(K)]
+        for row in ev_l:
+            for a_, b_ in row:
+                a_.record()
+                b_.record()
+        kv_l = kv_bytes_mean(K)
+        t_ms, h_ms = timed(lambda: step(stacked=False), K)
+        advance(K)
+        # the same once more with events around every layer's split kernel
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        host_issue = []
+        for s_ in range(min(K, 10)):
+            rope()
+            t_h = time.perf_counter()
+            attn(False, ev=ev_l[s_])
+            host_issue.append((time.perf_counter() - t_h) * 1e6 / NL)
+            accept()
+            append()
+            state["step"] += 1
+        torch.cuda.synchronize()
+        advance(min(K, 10))
+        dev_us = float(np.mean([a_.elapsed_time(b_) for row in ev_l[:min(K, 10)] for a_, b_ in row])) * 1e3
+        ideal_us = kv_l / NL / (achieved * 1e9) * 1e6      # what a layer's bytes take at the stacked launch's rate
+        per_layer = {"step_ms_layer_by_layer": t_ms, "step_ms_stacked": step_ms,
+                     "split_kernel_us_per_layer": dev_us,
+                     "device_fixed_us_per_layer_launch": dev_us - ideal_us,
+                     "host_issue_us_per_layer_call": float(np.mean(host_issue)),
+                     "note": "device fixed cost = a layer's own launch minus its bytes at the stacked launch's "
+                             "bandwidth; host = wall time of one memosight_attn_step call through the Python binding"}
+    elif n_phys > 1:
+        e_w = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+        for a_, b_ in e_w:
+            a_.record()
+            b_.record()
+        kv_w = kv_bytes_mean(K)
+        for s_ in range(K):
+            rope()
+            attn(True, ev=e_w[s_], rotate=False)
+            accept()
+            append(rotate=False)
+            state["step"] += 1
+        torch.cuda.synchronize()
+        advance(K)
+        w_ms = float(np.mean([a_.elapsed_time(b_) for a_, b_ in e_w]))
+        l2_warm = {"achieved": (kv_w + step_local) / (w_ms * 1e-3) / 1e9, "unit": "GB/s", "avg_launch_ms": w_ms,
+                   "note": "the same cache copy every step: it stays in the L2, not an HBM figure"}
+    # ---- the compaction event: every sequence ends a 512-token step (64 -> 8 + <o> for the tiny configuration)
+    seg, mem = (64, 8) if name == "tiny" else (SEG_LEN, MEM_TOKENS)
+    tail = mem + 1
+    lens_dev = inp.kv_len.clone()
+    can = all(L >= seg + tail for L in lens_now)
+    comp_us, comp_bytes = 0.0, 0
+    if can:
+        seg_len = torch.full((B,), seg, dtype=torch.int32, device=dev)
+        seg_start = (lens_dev - tail - seg).to(torch.int32)
+        ts = []
+        for _ in range(5):
+            inp.kv_len.copy_(lens_dev)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            ms.memosight_kv_compact(inp.k_cache, inp.v_cache, n_phys if NL > 1 else 1, lstride, stride, B, Hkv, D,
+                                    inp.kv_off, inp.kv_len, seg_start, seg_len, None, 0, tail)
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        lay = n_phys if NL > 1 else 1
+        comp_us = float(np.median(ts)) * 1e3 * (NL / lay)
+        comp_bytes = 2 * tail * Hkv * D * 2 * 2 * B * NL
+        assert inp.kv_len.cpu().tolist() == [L - seg for L in lens_now]
+        inp.kv_len.copy_(lens_dev)
+    gen_per_step = float(np.mean(keep))
+    parts = {"rope_us": part(0), "attn_us": part(1), "accept_us": part(2), "append_us": part(3),
+             "compaction_event_us": comp_us, "compaction_event_bytes": comp_bytes,
+             "compaction_event_gbs": (comp_bytes / (comp_us * 1e-6) / 1e9) if comp_us else None,
+             "compaction_amortised_us_per_step": comp_us * gen_per_step / seg,
+             "compaction_amortised_us_per_generated_token": comp_us / seg,
+             "note": f"event = all {B} sequences evict a {seg}-token step and keep {mem} memory tokens + <o>, all "
+                     f"{NL} layers" + (f" (measured on {n_phys} physical layers, scaled)" if NL > 1 else "") +
+                     f"; once per {seg} generated tokens of a sequence, {gen_per_step:.2f} tokens per step"}
+    line = {
+        "metric": METRIC_CONFIG, "value": T / (step_ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": K, "warmup": W,
+        "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": f"{cfg0.name}: H_q={Hq} H_kv={Hkv} D={D}, batch {B}, compacted KV "
+                               f"{cfg0.len_lo}..{cfg0.len_hi} (uniform from the seed; mean {np.mean(lens0):.0f}), "
+                               f"{cfg0.n_cand} candidate + d={cfg0.d} foresight rows per block, vocab {cfg0.vocab}, "
+                               f"{NL} logical layer(s) over {n_phys} physical cache layer(s)",
+                   "name": name, "global_batch": B, "layers": NL, "physical_layers": n_phys, "rows": rows,
+                   "n_cand": cfg0.n_cand, "d": cfg0.d,
+                   "l2": ("every layer's cache is far larger than the 126 MB L2; no flush" if layer_bytes > 4 * 126e6 else
+                          f"the cache of one layer ({layer_bytes / 1e6:.2f} MB) would sit in the L2: the steps rotate over "
+                          f"{n_phys} copies ({n_phys * layer_bytes / 1e6:.0f} MB) so that reads come from HBM")},
+        "kv_gb_per_step": kv_whole / 1e9, "host_issue_ms_per_step": host_ms,
+        "graph": {"ms_per_step": graph_ms, "value": T / (graph_ms * 1e-3), "unit": UNIT,
+                  "note": "K further steps captured once in a CUDA graph, one replay timed"},
+        "attention_only_tokens_per_s": T / (attn_ms * 1e-3), "roofline": roofline, "parts": parts, "clocks": clocks,
+        "gpu_launches": (1 + len(runs) + 1 + NL) * K if NL > 1 else 4 * K,
+    }
+    if per_layer:
+        line["per_layer"] = per_layer
+    if l2_warm:
+        line["l2_warm"] = l2_warm
+    if not args.no_cpu_baseline:
+        del inp, acc, q_all, ks_all, vs_all, out_all
+        torch.cuda.empty_cache()
+        cb = config_cpu_baseline(cfg0, name)
+        if name in ("tiny", "qwen7b"):
+            import subprocess
+            env = dict(os.environ, OMP_NUM_THREADS="1")
+            o = subprocess.run([sys.executable, os.path.abspath(__file__), "--config", name, "--cpu-only"], env=env,
+                               capture_output=True, text=True)
+            if o.returncode == 0:
+                one = json.loads(o.stdout.strip().splitlines()[-1])
+                cb["single_thread_value"] = one["value"]
+        line["cpu_baseline"] = cb
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------- the loop of Algorithm 1
+
+class DeviceToy:
+    """synth.ToyModel evaluated on the device with tensor operations (the same integer hashes, so
+    it predicts exactly what the host version predicts): stands in for the language model so that
+    the decoding loop runs without the host in the data path.  Not part of the library."""
+
+    def __init__(self, m, dev):
+        self.m, self.dev = m, dev
+
+    def _umod(self, h, n):
+        # h holds the bits of an unsigned 64-bit hash in an int64 lane: its value modulo n
+        r = torch.remainder(h, n)
+        return torch.where(h < 0, torch.remainder(r + ((1 << 64) % n), n), r)
+
+    def truth(self, b, pid, pid0):
+        m = self.m
+        key = b * 1000003 + pid
+        t = self._umod(synth.hash64(key, m.seed, synth.STREAM_TOY_TOKEN), m.vocab - 5)
+        t = torch.where(self._umod(synth.hash64(key, m.seed, synth.STREAM_TOY_DELIM), m.step_len) == 0,
+                        torch.full_like(t, m.tok_delim), t)
+        return torch.where(pid - pid0 >= m.eos_after, torch.full_like(t, m.tok_eos), t)
+
+    def predict(self, b, tok, pid, pid0):
+        m = self.m
+        t = self.truth(b, pid + 1, pid0)
+        miss = (tok == m.tok_f) & (self._umod(synth.hash64(b * 1000003 + pid, m.seed, synth.STREAM_TOY_HIT), 100)
+                                   >= m.hit_pct)
+        t = torch.where(miss, torch.remainder(t + 1, m.vocab - 5), t)
+        return torch.where(tok == m.tok_m, self._umod(synth.hash64(pid, m.seed, synth.STREAM_TOY_TOKEN), m.vocab - 5), t)
+
+
+class PlantedLogits:
+    """fp32 [rows][V] seeded noise with one winner per row planted 40 above it; the winners move
+    from step to step by undoing the last plant and making the next (four small index kernels)."""
+
+    def __init__(self, rows, V, seed, dev):
+        self.buf = synth.normal_f32(rows * V, seed, synth.STREAM_LOGITS, 2.0, device=dev).view(rows, V)
+        self.rows = torch.arange(rows, device=dev)
+        self.col = torch.zeros(rows, dtype=torch.int64, device=dev)
+        self.noise = self.buf[self.rows, self.col].clone()
+
+    def plant(self, col):
+        self.buf[self.rows, self.col] = self.noise          # undo
+        self.col.copy_(col)
+        self.noise.copy_(self.buf[self.rows, self.col])
+        self.buf[self.rows, self.col] = self.noise + 40.0
+
+
+def run_loop(args, ms, dev):
+    """Secondary workload: the whole inference loop of Algorithm 1 on device-resident state --
+    Predict+Verify blocks until a step ends, then the compression block (memory tokens + <o>
+    through the large-block kernel), append and eviction -- with a toy model as the logits source.
+    Per iteration the host reads one 16-byte summary (rows, live sequences, sequences waiting for
+    compression); everything else stays on the device.  Every iteration is one CUDA graph replay
+    (a step graph or a compression graph, each ending with the plan of the next block)."""
+    import ctypes as C
+    assert int(os.environ.get("WORLD_SIZE", "1")) == 1
+    Hq, Hkv, D, NL = 32, 8, 128, max(1, args.layers or 1)
+    V, L0, max_mem, max_out = 128256, 1024, 64, 1500
+    base = 5.0e5
+    results = []
+    grid = [(B, d, c) for B in ((args.batch,) if args.batch != 128 else (1, 64)) for c in (3, 5) for d in range(0, 5)]
+    if args.d != 3:
+        grid = [(B, d, c) for (B, d, c) in grid if d == args.d]
+    for (B, d, c) in grid:
+        m = synth.ToyModel(vocab=V, hit_pct=60, step_len=23, eos_after=1200, seed=0x70F0 + B)
+        toy = DeviceToy(m, dev)
+        pid0 = [L0 + 3 * b for b in range(B)]
+        cap = L0 + 1400
+        n_slots = B * cap
+        stride, lstride = n_slots * D, Hkv * n_slots * D
+        k_cache = synth.normal_bf16(NL * lstride, 11, synth.STREAM_KCACHE, device=dev).view(NL, Hkv, n_slots, D)
+        v_cache = synth.normal_bf16(NL * lstride, 11, synth.STREAM_VCACHE, device=dev).view(NL, Hkv, n_slots, D)
+        i32 = lambda x: torch.tensor(x, dtype=torch.int32, device=dev)
+        g_off = torch.tensor([b * cap for b in range(B)], dtype=torch.int64, device=dev)
+        g_len, g_cap = i32([L0] * B), i32([cap] * B)
+        first = [m.truth(b, pid0[b], pid0[b]) for b in range(B)]
+        cand = torch.zeros((B, d + 1), dtype=torch.int32, device=dev)
+        cand[:, 0] = i32(first)
+        st_t = dict(kv_len=g_len, pos_next=i32(pid0), seg_start=i32([L0] * B), seg_n=i32([0] * B), seg_pid0=i32(pid0),
+                    cand=cand, n_cand=i32([1] * B), flags=i32([0] * B),
+                    out_tok=torch.zeros((B, max_out), dtype=torch.int32, device=dev), n_out=i32([0] * B))
+        st = ms.decode_state(B, d, c, max_out, max_mem, m.tok_f, m.tok_m, m.tok_o, m.tok_delim, m.tok_eos, **st_t)
+        nq_s, nq_c = 2 * d + 1, max_mem + 1
+        Ts, Tc = B * nq_s, B * nq_c
+        q_off, n_blk = torch.zeros(B + 1, dtype=torch.int32, device=dev), torch.zeros(B, dtype=torch.int32, device=dev)
+        row_tok, pos_id, draft = (torch.zeros(Tc, dtype=torch.int32, device=dev) for _ in range(3))
+        n_keep, seg_s, seg_l = (torch.zeros(B, dtype=torch.int32, device=dev) for _ in range(3))
+        summary = torch.zeros(4, dtype=torch.int32, device=dev)
+        h_summary = torch.zeros(4, dtype=torch.int32).pin_memory()
+        scratch = torch.empty(ms.memosight_decode_scratch_bytes(B), dtype=torch.uint8, device=dev)
+        am, nm = torch.zeros(Tc + 1, dtype=torch.int32, device=dev), torch.zeros(B, dtype=torch.int32, device=dev)
+        am_o = torch.zeros(B, dtype=torch.int32, device=dev)
+        overflow = torch.zeros(1, dtype=torch.int32, device=dev)
+        aws = torch.empty(ms.memosight_accept_workspace_bytes(max(Ts, B), V), dtype=torch.uint8, device=dev)
+        # q / k / v of the blocks: fixed seeded tensors (what the attention computes does not steer the toy model)
+        q = synth.normal_bf16(NL * Tc * Hq * D, 12, synth.STREAM_Q, device=dev).view(NL, Tc, Hq, D)
+        ks = synth.normal_bf16(NL * Tc * Hkv * D, 12, synth.STREAM_KSTEP, device=dev).view(NL, Tc, Hkv, D)
+        vs = synth.normal_bf16(NL * Tc * Hkv * D, 12, synth.STREAM_VSTEP, device=dev).view(NL, Tc, Hkv, D)
+        out = torch.empty((NL, Tc, Hq, D), dtype=torch.bfloat16, device=dev)
+        max_kv = cap
+        wsb_s = ms.memosight_attn_workspace_bytes(B, Hq, Hkv, D, max_kv, nq_s)
+        wsb_c = ms.memosight_attn_workspace_bytes(B, Hq, Hkv, D, max_kv, nq_c)
+        ws_s = torch.empty(wsb_s, dtype=torch.uint8, device=dev)
+        ws_c = torch.empty(wsb_c, dtype=torch.uint8, device=dev)
+        lg_s, lg_c = PlantedLogits(Ts, V, 13, dev), PlantedLogits(B, V, 14, dev)
+        pid0_t = torch.tensor(pid0, dtype=torch.int64, device=dev)
+        rows_s = torch.arange(Ts, device=dev, dtype=torch.int32)
+        row_off_c = torch.arange(B + 1, dtype=torch.int32, device=dev)
+        draft_c = torch.full((B,), -1, dtype=torch.int32, device=dev)
+        nm_c = torch.zeros(B, dtype=torch.int32, device=dev)
+        n_iter_cap = 4000
+        len_log = torch.zeros((n_iter_cap, B), dtype=torch.int32, device=dev)
+
+        def attn_params(layer, ws, wsb, max_nq, T):
+            return ms.attn_params(batch=B, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, k_cache=k_cache[layer],
+                                  v_cache=v_cache[layer], kv_head_stride=stride, n_slots=n_slots, kv_off=g_off,
+                                  kv_len=g_len, max_kv_len=max_kv, max_nq=max_nq, q_off=q_off, n_cand=n_blk, anchor=None,
+                                  total_rows=T, sm_scale=0.0, q=q[layer], k_step=ks[layer], v_step=vs[layer],
+                                  out=out[layer], lse=None, workspace=ws, workspace_bytes=wsb)
+        ap_s = [attn_params(l, ws_s, wsb_s, nq_s, Ts) for l in range(NL)]
+        ap_c = [attn_params(l, ws_c, wsb_c, nq_c, Tc) for l in range(NL)]
+
+        def plan():
+            ms.memosight_decode_plan(st, q_off, n_blk, row_tok, pos_id, draft, summary, scratch)
+            h_summary.copy_(summary, non_blocking=True)
+
+        def step_body():
+            # one Predict+Verify block of every live sequence (rows beyond q_off[B] hold stale, harmless data)
+            for l in range(NL):
+                ms.memosight_rope_qk(q[l], ks[l], pos_id, Ts, Hq, Hkv, D, base)
+                ms.memosight_attn_step(ap_s[l])
+            seq = torch.searchsorted(q_off[1:], rows_s, right=True).clamp_(max=B - 1).to(torch.int64)
+            win = toy.predict(seq, row_tok[:Ts].to(torch.int64), pos_id[:Ts].to(torch.int64), pid0_t[seq])
+            lg_s.plant(win)
+            ms.memosight_accept(lg_s.buf, V, V, q_off, B, Ts, draft, am, nm, None, aws, aws.numel())
+            ms.memosight_decode_commit(st, q_off, am, nm, n_keep)
+            for l in range(NL):
+                ms.memosight_kv_append(k_cache[l], v_cache[l], stride, n_slots, B, Hkv, D, g_off, g_len, g_cap, ks[l],
+                                       vs[l], q_off, n_blk, n_keep, nq_s, l == NL - 1, overflow)
+            plan()
+
+        def compress_body():
+            ms.memosight_decode_plan_compress(st, q_off, n_blk, row_tok, pos_id, n_keep, seg_s, seg_l, summary, scratch)
+            for l in range(NL):
+                ms.memosight_rope_qk(q[l], ks[l], pos_id, Tc, Hq, Hkv, D, base)
+                ms.memosight_attn_step(ap_c[l])
+            # the model's head is only needed on <o>, the last row of each block: one logits row per sequence
+            last = (q_off[1:].to(torch.int64) - 1).clamp_(min=0)
+            bs = torch.arange(B, device=dev, dtype=torch.int64)
+            win = toy.predict(bs, row_tok[last].to(torch.int64), pos_id[last].to(torch.int64), pid0_t)
+            lg_c.plant(win)
+            ms.memosight_accept(lg_c.buf, V, V, row_off_c, B, B, draft_c, am_o, nm_c, None, aws, aws.numel())
+            # to the block's last row, where commit_compress reads it (sequences without a block: a spare slot)
+            am[torch.where(q_off[1:] > q_off[:-1], last, torch.full_like(last, Tc))] = am_o
+            for l in range(NL):
+                ms.memosight_kv_append(k_cache[l], v_cache[l], stride, n_slots, B, Hkv, D, g_off, g_len, g_cap, ks[l],
+                                       vs[l], q_off, n_blk, n_keep, nq_c, l == NL - 1, overflow)
+            ms.memosight_kv_compact(k_cache, v_cache, NL, lstride, stride, B, Hkv, D, g_off, g_len, seg_s, seg_l, None,
+                                    0, max_mem + 1)
+            ms.memosight_decode_commit_compress(st, q_off, am)
+            plan()
+
+        # warm both bodies up on a scratch copy of the state?  They mutate it, so instead: run the
+        # first iterations eagerly (they are part of the decode), then capture and replay
+        side = torch.cuda.Stream()
+        graphs = {}
+
+        def run(body, name, use_graph):
+            if not use_graph:
+                body()
+                return
+            if name not in graphs:
+                g = torch.cuda.CUDAGraph()
+                torch.cuda.synchronize()
+                with torch.cuda.graph(g, stream=side):
+                    body()
+                graphs[name] = g
+            graphs[name].replay()
+
+        plan()
+        torch.cuda.synchronize()
+        steps = comps = iters = 0
+        eager_iters = {"step": 0, "compress": 0}
+        t_start = None
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n_timed_steps = n_timed_comps = 0
+        tokens_at_start = 0
+        while True:
+            T, live, pending, _ = h_summary.tolist()
+            if T == 0 and pending == 0:
+                break
+            name = "compress" if pending else "step"
+            use_graph = eager_iters[name] >= 2            # two eager runs of a body first (set-up, caches)
+            if not use_graph:
+                eager_iters[name] += 1
+            elif t_start is None and all(v >= 2 for v in eager_iters.values()) and len(graphs) == 2:
+                torch.cuda.synchronize()
+                t_start = time.perf_counter()
+                e0.record()
+                tokens_at_start = int(st_t["n_out"].sum().item())
+            run(compress_body if pending else step_body, name, use_graph)
+            len_log[min(iters, n_iter_cap - 1)].copy_(g_len)
+            torch.cuda.synchronize()                      # the 16-byte summary of the next block is on the host
+            if t_start is not None:
+                if pending:
+                    n_timed_comps += 1
+                else:
+                    n_timed_steps += 1
+            steps += 0 if pending else 1
+            comps += 1 if pending else 0
+            iters += 1
+            assert iters < n_iter_cap
+        e1.record()
+        torch.cuda.synchronize()
+        wall = time.perf_counter() - (t_start or time.perf_counter())
+        assert int(overflow.item()) == 0, "a sequence outgrew its cache region"
+        # the accepted tokens are what plain token-by-token greedy decoding with the same model gives
+        n_out = st_t["n_out"].cpu().tolist()
+        out_tok = st_t["out_tok"].cpu()
+        for b in range(min(B, 4)):
+            want, pid, tok = [], pid0[b], first[b]
+            while len(want) < max_out:
+                want.append(tok)
+                if tok == m.tok_eos:
+                    break
+                if tok == m.tok_delim:
+                    tok, pid = m.predict(b, m.tok_o, pid + 1, pid0[b]), pid + 2
+                else:
+                    tok, pid = m.predict(b, tok, pid, pid0[b]), pid + 1
+            assert out_tok[b, :min(n_out[b], max_out)].tolist() == want[:min(n_out[b], max_out)], f"sequence {b} is not greedy"
+        total_tokens = int(sum(min(n, max_out) for n in n_out))
+        timed_tokens = total_tokens - tokens_at_start
+        lens = len_log[:iters].float().mean(dim=1).cpu().tolist()
+        pick = [lens[int(i * (len(lens) - 1) / 9)] for i in range(10)] if lens else []
+        line = {
+            "metric": "Predict+Verify steps/s of the whole inference loop (Algorithm 1) on device-resident state",
+            "value": n_timed_steps / wall if wall > 0 else 0.0, "unit": "steps/s", "n_gpus": 1,
+            "steps": n_timed_steps, "warmup": steps - n_timed_steps, "ms_per_step": wall / max(n_timed_steps, 1) * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"loop: 8B-shape attention ({NL} layer(s)), batch {B}, d={d} foresight tokens, "
+                                   f"compression ratio c={c}, prompt cache {L0}, toy model (60 % foresight hit rate, "
+                                   f"reasoning steps of ~23 tokens, <eos> after 1200 positions), vocab {V}",
+                       "global_batch": B, "d": d, "c": c, "layers": NL},
+            "accepted_tokens_per_s": timed_tokens / wall if wall > 0 else 0.0,
+            "tokens_per_step": timed_tokens / max(n_timed_steps, 1) / B,
+            "compressions": comps, "timed_compressions": n_timed_comps, "iterations": iters,
+            "device_ms_timed": e0.elapsed_time(e1) if t_start is not None else None,
+            "mean_cache_length_over_time": [round(x, 1) for x in pick],
+            "peak_mean_cache_length": max(lens) if lens else None,
+            "uncompressed_length_at_end": L0 + float(np.mean([min(n, max_out) for n in n_out])),
+            "note": "one CUDA graph replay and one 16-byte device-to-host read per iteration; wall-clock time",
+        }
+        results.append(line)
+        print(json.dumps(line), flush=True)
+        del k_cache, v_cache, q, ks, vs, out, lg_s, lg_c, graphs
+        torch.cuda.empty_cache()
+    print("| batch | d | c | steps/s | accepted tokens/s | tokens per step and sequence | ms per step | compressions | "
+          "mean cache length start -> peak -> end | uncompressed length at the end |")
+    print("|---:|---:|---:|---:|---:|---:|---:|---:|---|---:|")
+    for j in results:
+        c_ = j["config"]
+        tr = j["mean_cache_length_over_time"]
+        print(f"| {c_['global_batch']} | {c_['d']} | {c_['c']} | {j['value']:.0f} | {j['accepted_tokens_per_s']:.0f} | "
+              f"{j['tokens_per_step']:.2f} | {j['ms_per_step']:.3f} | {j['compressions']} | "
+              f"{tr[0]:.0f} -> {j['peak_mean_cache_length']:.0f} -> {tr[-1]:.0f} | {j['uncompressed_length_at_end']:.0f} |")
+
+
+# --------------------------------------------------------------------------- the small HBM-bound kernels
+
+def run_cacheops(args, ms, dev):
+    """Secondary workload: the HBM-bound kernels around the attention, each timed alone on the
+    long-CoT shapes -- the compaction event (512 -> 170 + <o>, every sequence, every layer), an
+    eviction by keep list (every third of the last 3000 entries dropped: short runs; and a
+    window-plus-prefix keep set: long runs), RoPE and append of the compression block's 171 tokens
+    per sequence, and the split-KV merge of a small batch.  Bytes are the algorithmic ones: moved
+    entries x 2 (read + write) for the cache operations, one read + one write of q and k for RoPE."""
+    B = args.batch if args.batch != 128 else 64
+    NL = args.layers or 4
+    Hq, Hkv, D = 32, 8, 128
+    reps = max(3, min(args.steps, 20))
+    cfg = synth.StepConfig("cacheops", B, Hq, Hkv, D, 9000, 12000, 4, 4, 5e5, 100, n_layers=NL, seed=78)
+    inp = synth.make_step_inputs(cfg, device=dev)
+    stride, lstride = inp.n_slots * D, Hkv * inp.n_slots * D
+    len0 = inp.kv_len.clone()
+    peak, peak_kind = peak_hbm()
+
+    def timeit(f, reset):
+        for _ in range(2):
+            reset()
+            f()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(reps):
+            reset()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            f()
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        return float(np.median(ts))
+
+    rows = []
+
+    def report(name, kernel, ms_, nbytes, what):
+        gbs = nbytes / (ms_ * 1e-3) / 1e9
+        rows.append({"name": name, "kernel": kernel, "us": ms_ * 1e3, "algorithmic_bytes": nbytes, "achieved": gbs,
+                     "unit": "GB/s", "frac": gbs / peak, "frac_of_nominal_8000": gbs / 8000.0, "what": what})
+
+    reset = lambda: inp.kv_len.copy_(len0)
+    # ---- compaction event
+    tail = MEM_TOKENS + 1
+    seg_start = (len0 - tail - SEG_LEN).to(torch.int32)
+    seg_len = torch.full((B,), SEG_LEN, dtype=torch.int32, device=dev)
+    t = timeit(lambda: ms.memosight_kv_compact(inp.k_cache, inp.v_cache, NL, lstride, stride, B, Hkv, D, inp.kv_off,
+                                               inp.kv_len, seg_start, seg_len, None, 0, tail), reset)
+    report("compaction event", "kv_compact_move_kernel", t, 2 * tail * Hkv * D * 2 * 2 * B * NL,
+           f"{B} sequences x {NL} layers evict a {SEG_LEN}-token step, {tail} entries slide down")
+    # ---- eviction by keep list
+    lens = len0.cpu().tolist()
+    for label, keep_fn in (("every third of the last 3000 dropped", lambda L: [i for i in range(L) if i < L - 3000 or i % 3]),
+                           ("first 384 + last 4096 kept", lambda L: list(range(384)) + list(range(L - 4096, L)))):
+        keep = [keep_fn(L) for L in lens]
+        max_keep = max(len(k) for k in keep)
+        ki = torch.zeros((B, max_keep), dtype=torch.int32)
+        for b in range(B):
+            ki[b, :len(keep[b])] = torch.tensor(keep[b], dtype=torch.int32)
+        ki = ki.to(dev)
+        nk = torch.tensor([len(k) for k in keep], dtype=torch.int32, device=dev)
+        t = timeit(lambda: ms.memosight_kv_gather(inp.k_cache, inp.v_cache, NL, lstride, stride, B, Hkv, D, inp.kv_off,
+                                                  inp.kv_len, ki, max_keep, nk, max_keep), reset)
+        moved = sum(sum(1 for j, i in enumerate(k) if i != j) for k in keep)
+        report(f"keep-list eviction ({label})", "kv_gather_kernel", t, moved * NL * 2 * Hkv * D * 2 * 2,
+               f"{moved} entries per layer change their slot")
+    reset()
+    # ---- RoPE and append of the compression blocks
+    nq = tail
+    T = B * nq
+    q = synth.normal_bf16(T * Hq * D, 5, synth.STREAM_Q, device=dev).view(T, Hq, D)
+    k = synth.normal_bf16(T * Hkv * D, 5, synth.STREAM_KSTEP, device=dev).view(T, Hkv, D)
+    pos = torch.from_numpy(np.concatenate([
+        np.concatenate([ms.memosight_upl_pids(3 * L, SEG_LEN, 3)[:MEM_TOKENS], [ms.memosight_out_pid(3 * L, SEG_LEN)]])
+        for L in lens]).astype(np.int32)).to(dev)
+    t = timeit(lambda: ms.memosight_rope_qk(q, k, pos, T, Hq, Hkv, D, 5e5), lambda: None)
+    report("RoPE of the compression blocks", "rope_qk_kernel", t, T * (Hq + Hkv) * D * 2 * 2,
+           f"{T} tokens at UPL position IDs, in place")
+    q_off = torch.arange(0, T + 1, nq, dtype=torch.int32, device=dev)
+    n_c = torch.full((B,), nq, dtype=torch.int32, device=dev)
+    # (the append keeps the lengths: bump_len = 0, so every repetition writes the same slots)
+    t = timeit(lambda: ms.memosight_kv_append(inp.k_cache[0], inp.v_cache[0], stride, inp.n_slots, B, Hkv, D,
+                                              inp.kv_off, inp.kv_len, None, k, k, q_off, n_c, n_c, nq, 0), lambda: None)
+    report("append of the compression blocks (one layer)", "kv_append_kernel", t, T * Hkv * D * 2 * 2 * 2,
+           f"{nq} rows per sequence, K and V")
+    # ---- the merge of a small batch (every unit cut across many CTAs)
+    Bs, d = 2, 7
+    scfg = synth.sweep(Bs, d, 16384, True)
+    sinp = synth.make_step_inputs(scfg, device=dev)
+    Ts = Bs * scfg.n_q
+    out = torch.empty((Ts, Hq, D), dtype=torch.bfloat16, device=dev)
+    wsb = ms.memosight_attn_workspace_bytes(Bs, Hq, Hkv, D, 16384, scfg.n_q)
+    ws = torch.empty(wsb, dtype=torch.uint8, device=dev)
+    ap = ms.attn_params(batch=Bs, n_q_heads=Hq, n_kv_heads=Hkv, head_dim=D, k_cache=sinp.k_cache[0],
+                        v_cache=sinp.v_cache[0], kv_head_stride=sinp.n_slots * D, n_slots=sinp.n_slots,
+                        kv_off=sinp.kv_off, kv_len=sinp.kv_len, max_kv_len=16384, max_nq=scfg.n_q, q_off=sinp.q_off,
+                        n_cand=sinp.n_cand, anchor=None, total_rows=Ts, sm_scale=0.0, q=sinp.q, k_step=sinp.k_step,
+                        v_step=sinp.v_step, out=out, lse=None, workspace=ws, workspace_bytes=wsb)
+    ev = (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+    for e in ev:
+        e.record()
+    ms.memosight_attn_debug_events(ev[0].cuda_event, ev[1].cuda_event)
+    t_all = timeit(lambda: ms.memosight_attn_step(ap), lambda: None)
+    torch.cuda.synchronize()
+    t_split = ev[0].elapsed_time(ev[1])
+    ms.memosight_attn_debug_events(None, None)
+    n_sm = torch.cuda.get_device_properties(dev).multi_processor_count
+    rows_p = scfg.n_q * (Hq // Hkv)
+    report("split-KV merge of a small batch (call minus split kernel)", "attn_merge_kernel", max(t_all - t_split, 1e-6),
+           n_sm * rows_p * (D + 2) * 4 + Ts * Hq * D * 2,
+           f"batch {Bs}, d={d}: {Bs * Hkv} units x {rows_p} rows, one partial per CTA ({n_sm}); latency-bound")
+    line = {"metric": "GB/s of the HBM-bound kernels around the attention (algorithmic bytes / device time)",
+            "unit": "GB/s", "n_gpus": 1, "steps": reps, "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"cache operations on long-CoT shapes: batch {B}, {NL} layers, caches 9000..12000, "
+                                   f"8B shape", "global_batch": B, "layers": NL},
+            "peak": peak, "peak_source": f"{peak_kind} copy bandwidth", "kernels": rows}
+    print(json.dumps(line), flush=True)
+    print("| operation | kernel | µs | algorithmic MB | GB/s | of measured HBM | of 8 TB/s |")
+    print("|---|---|---:|---:|---:|---:|---:|")
+    for r in rows:
+        print(f"| {r['name']} | {r['kernel']} | {r['us']:.1f} | {r['algorithmic_bytes'] / 1e6:.1f} | {r['achieved']:.0f} | "
+              f"{r['frac']:.2f} | {r['frac_of_nominal_8000']:.2f} |")
 
 
 def peak_tensor():

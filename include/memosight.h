@@ -250,6 +250,18 @@ MS_API int32_t memosight_attn_debug_events(void* ev_split_begin, void* ev_split_
  * (its output is then undefined).  Meant for tests and debugging. */
 MS_API int32_t memosight_attn_status(const void* workspace, memosight_stream_t stream);
 
+/* Diagnostics of the bounded waits.  Every wait inside the kernels (on an mbarrier that a bulk
+ * copy or a tensor-core operation completes) gives up after a limit, 4 s by default; the kernel
+ * then records it, drains what it has in flight and returns (see memosight_attn_status).
+ * memosight_debug_set_wait_limit_us changes that limit for the launches that follow,
+ * process-wide, and returns the previous one (0 only queries).  memosight_debug_wait_timeout
+ * queues a one-warp kernel that waits, with a limit of limit_us (at most one second), on a
+ * barrier at which nobody arrives: the wait runs out, the kernel returns, and
+ * memosight_attn_status(workspace) then reports MS_ERR_DEVICE_TIMEOUT once -- the whole failure
+ * path exercised without anything failing.  workspace: device, 256-byte aligned, >= 256 bytes. */
+MS_API uint32_t memosight_debug_set_wait_limit_us(uint32_t limit_us);
+MS_API int32_t memosight_debug_wait_timeout(void* workspace, uint32_t limit_us, memosight_stream_t stream);
+
 /* ---- KV compaction and append (Sec. 2.1.2; Algorithm 1: UpdateCache, S <- S (+) A) ------- */
 
 /* Evicts one verbose step per sequence from every layer's K and V cache, in place:
@@ -447,7 +459,10 @@ MS_API int32_t memosight_decode_commit_compress(const memosight_decode_state* st
  * into `stream` before the accept; calls for one device share that stream and the
  * events, so issue them one after the other, not from several threads at once,
  * and make the first call on a device outside any stream capture.
- * The call returns after queueing; synchronise `stream` before reading h_*. */
+ * The call returns after queueing; synchronise `stream` before reading h_*.
+ * Any h_* pointer may be NULL: that tensor is then taken from (or left in) its device staging
+ * buffer and not copied.  With all of them NULL the call is the whole device-resident step --
+ * RoPE, attention, accept, append, compaction -- queued by one call into the library. */
 typedef struct memosight_step_host_params {
   uint32_t struct_size;          /* sizeof(memosight_step_host_params)                         */
   memosight_attn_params attn;    /* device-side description of the step: q, k_step, v_step, out,

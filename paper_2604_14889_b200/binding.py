@@ -142,6 +142,10 @@ def lib() -> C.CDLL:
         L.memosight_attn_step_layers.argtypes = [C.POINTER(AttnParams), C.POINTER(AttnLayers), C.c_void_p]
         L.memosight_attn_debug_events.restype = C.c_int32
         L.memosight_attn_debug_events.argtypes = [C.c_void_p, C.c_void_p]
+        L.memosight_debug_set_wait_limit_us.restype = C.c_uint32
+        L.memosight_debug_set_wait_limit_us.argtypes = [C.c_uint32]
+        L.memosight_debug_wait_timeout.restype = C.c_int32
+        L.memosight_debug_wait_timeout.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p]
         L.memosight_attn_set_path.restype = C.c_int32
         L.memosight_attn_set_path.argtypes = [C.c_int32]
         L.memosight_attn_status.restype = C.c_int32
@@ -326,6 +330,17 @@ def memosight_attn_set_path(path: int) -> int:
     if rc < 0:
         raise MemosightError(rc, "memosight_attn_set_path")
     return rc
+
+
+def memosight_debug_set_wait_limit_us(limit_us: int) -> int:
+    """Limit of one bounded device-side wait for later launches; returns the previous one (0 only queries)."""
+    return int(lib().memosight_debug_set_wait_limit_us(int(limit_us)))
+
+
+def memosight_debug_wait_timeout(workspace, limit_us: int, stream=None) -> None:
+    """Queues the one-warp kernel whose bounded wait runs out after limit_us microseconds."""
+    _check(int(lib().memosight_debug_wait_timeout(_ptr(workspace), int(limit_us), _stream(stream))),
+           "memosight_debug_wait_timeout")
 
 
 def memosight_attn_status(workspace, stream=None) -> int:

@@ -186,7 +186,7 @@ __device__ __forceinline__ void accept_tail(const Tail& t, const Cand* part, int
 
 __global__ void __launch_bounds__(kStreamThreads, 1)
 argmax_stream_kernel(const float* __restrict__ logits, int64_t ld_v, int V, int n_chunks, int n_items,
-                     Cand* __restrict__ part, const Tail tail) {
+                     Cand* __restrict__ part, const Tail tail, unsigned int wait_limit_us) {
   extern __shared__ __align__(1024) uint8_t smem[];
   const uint32_t sb = ms::smem_u32(smem);
   const uint32_t bars = sb + kStages * kStageBytes;           // full[kStages], empty[kStages]
@@ -197,7 +197,7 @@ argmax_stream_kernel(const float* __restrict__ logits, int64_t ld_v, int V, int 
       ms::mbar_init(bars + 8 * i, 1);
       ms::mbar_init(bars + 8 * (kStages + i), 1);
     }
-    *abort_flag = 0;
+    ms::wait_ctx_init(abort_flag, wait_limit_us);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
@@ -370,7 +370,8 @@ int32_t launch_accept(const float* logits, int64_t ld_v, int vocab, const int32_
       if (sms <= 0) return ms::cuda_status(cudaErrorNoDevice);
       if (total_rows < ms::kDoneBankWords && batch <= kTailMaxBatch) tail.cnt = ms::done_bank(part);
       MS_CUDA_TRY(ms::launch_pdl(argmax_stream_kernel, dim3(n_items < sms ? n_items : sms), dim3(kStreamThreads),
-                                 kStreamSmem, st, logits, ld_v, vocab, n_chunks, n_items, part, tail));
+                                 kStreamSmem, st, logits, ld_v, vocab, n_chunks, n_items, part, tail,
+                                 ms::wait_limit_us()));
       if (tail.cnt) return MS_OK;
     } else if (vec) {
       argmax_chunks_kernel<true><<<static_cast<unsigned>(n_items), kThreads, 0, st>>>(logits, ld_v, vocab, n_chunks, part);

@@ -1,8 +1,14 @@
 // Status strings, error bookkeeping and the host-only position-layout helpers
 // (AMA, UPL, <o> and step-block PIDs; paper Sec. 2.1.2 and Sec. 2.2).
+#include <atomic>
+
 #include "common.cuh"
 
 namespace ms {
+
+static std::atomic<unsigned int> g_wait_limit_us{4000000u};
+
+unsigned int wait_limit_us() { return g_wait_limit_us.load(std::memory_order_relaxed); }
 
 static thread_local int32_t g_last_cuda_error = 0;
 
@@ -40,6 +46,11 @@ const char* memosight_status_string(int32_t status) {
 }
 
 int32_t memosight_last_cuda_error(void) { return ms::g_last_cuda_error; }
+
+uint32_t memosight_debug_set_wait_limit_us(uint32_t limit_us) {
+  if (limit_us == 0) return ms::g_wait_limit_us.load(std::memory_order_relaxed);
+  return ms::g_wait_limit_us.exchange(limit_us, std::memory_order_relaxed);
+}
 
 // l = ceil(n / c)  (Sec. 2.1.2, Adaptive Memory Allocation)
 int32_t memosight_ama(int32_t n, int32_t c) {

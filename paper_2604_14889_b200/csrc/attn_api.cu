@@ -3,7 +3,7 @@
 #include <math.h>
 #include <stddef.h>
 
-#include "attn_internal.cuh"
+#include "attn_sched.cuh"
 
 #include <atomic>
 #include <mutex>
@@ -250,6 +250,7 @@ int32_t attn_call(const memosight_attn_params* p, const memosight_attn_layers* l
   a.n_layers = 1;
   a.kv_layer_stride = a.q_layer_stride = a.kstep_layer_stride = a.out_layer_stride = a.lse_layer_stride = 0;
   a.done = nullptr;
+  a.wait_limit_us = ms::wait_limit_us();
   a.ev_split_begin = t_ev_begin;
   a.ev_split_end = t_ev_end;
 
@@ -299,6 +300,32 @@ extern "C" int32_t memosight_attn_step_layers(const memosight_attn_params* p, co
                                               memosight_stream_t stream) {
   if (!layers) return MS_ERR_INVALID_ARG;
   return attn_call(p, layers, stream);
+}
+
+namespace {
+
+// One warp waits, with the bounded wait every kernel of the library uses, on a barrier at which
+// nobody ever arrives: the wait runs into its limit, records that in the status word and returns.
+__global__ void wait_probe_kernel(uint32_t* status, unsigned int limit_us) {
+  __shared__ __align__(8) unsigned long long bar;
+  __shared__ int ctx[2];
+  if (threadIdx.x == 0) {
+    ms::mbar_init(ms::smem_u32(&bar), 1);
+    ms::wait_ctx_init(ctx, limit_us);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  (void)ms::mbar_wait(ms::smem_u32(&bar), 0, ctx, status);
+}
+
+}  // namespace
+
+extern "C" int32_t memosight_debug_wait_timeout(void* workspace, uint32_t limit_us, memosight_stream_t stream) {
+  if (!workspace || limit_us == 0 || limit_us > 1000000u) return MS_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255u) return MS_ERR_ALIGNMENT;
+  wait_probe_kernel<<<1, 32, 0, ms::as_stream(stream)>>>(static_cast<uint32_t*>(workspace), limit_us);
+  MS_LAUNCH_CHECK();
+  return MS_OK;
 }
 
 extern "C" int32_t memosight_attn_status(const void* workspace, memosight_stream_t stream) {

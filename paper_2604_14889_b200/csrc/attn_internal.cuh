@@ -37,6 +37,7 @@ struct AttnArgs {
   // Counters of the in-kernel merge (two per persistent CTA, zero between launches), or NULL:
   // the merge is then a launch of its own.
   unsigned int* done;
+  unsigned int wait_limit_us;   // limit of one bounded device-side wait
   cudaEvent_t ev_split_begin, ev_split_end;   // optional timing events around the split kernel
 };
 

@@ -143,7 +143,7 @@ attn_split_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
       mbar_init(bar_empty + 8 * s, kConsumerWarps);
     }
     mbar_init(bar_merge, kConsumerWarps);
-    *abort_flag = 0;
+    wait_ctx_init(abort_flag, a.wait_limit_us);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();   // prefix consumed, barriers initialised: stage memory may now be filled

@@ -10,7 +10,17 @@ namespace ms {
 
 constexpr int kTile = 128;                 // keys per pipeline stage
 constexpr uint32_t kTimeoutMagic = 0x4D535431u;
-constexpr unsigned long long kWaitLimitNs = 4000000000ull;
+constexpr unsigned int kWaitLimitDefaultUs = 4000000u;   // 4 s: far beyond anything but a dead device
+
+// Every bounded wait of a CTA shares two shared-memory words: [0] the abort flag, [1] the limit of
+// one wait in microseconds (a launch parameter, see wait_limit_us()).
+__device__ __forceinline__ void wait_ctx_init(volatile int* ctx, unsigned int limit_us) {
+  ctx[0] = 0;
+  ctx[1] = static_cast<int>(limit_us);
+}
+__device__ __forceinline__ unsigned long long wait_limit_ns(volatile int* ctx) {
+  return static_cast<unsigned long long>(static_cast<unsigned int>(ctx[1])) * 1000ull;
+}
 
 // ---------------------------------------------------------------- PTX wrappers
 
@@ -47,12 +57,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // then records the timeout in the workspace status word and raises the abort flag).
 static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                             uint32_t* status) {
-  const unsigned long long t0 = global_ns();
+  const unsigned long long t0 = global_ns(), limit = wait_limit_ns(abort_flag);
   for (uint32_t spin = 1;; ++spin) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((spin & 63u) == 0) {
       if (*abort_flag) return false;
-      if (global_ns() - t0 > kWaitLimitNs) {
+      if (global_ns() - t0 > limit) {
         *abort_flag = 1;
         atomicExch(status, kTimeoutMagic);
         return false;

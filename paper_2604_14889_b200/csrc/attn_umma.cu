@@ -169,7 +169,7 @@ attn_umma_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
       mbar_init(bars + 8 * (kBarPvDone + i), 1);
     }
     mbar_init(bars + 8 * kBarDrain, 1);
-    *abort_flag = 0;
+    wait_ctx_init(abort_flag, a.wait_limit_us);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();   // the prefix has been consumed
@@ -311,7 +311,7 @@ attn_umma_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
       // aborting: let the tensor pipe run dry before tensor memory is released
       umma_commit(bars + 8 * kBarDrain);
       const unsigned long long t_begin = global_ns();
-      while (!mbar_try_wait(bars + 8 * kBarDrain, 0) && global_ns() - t_begin < kWaitLimitNs) {
+      while (!mbar_try_wait(bars + 8 * kBarDrain, 0) && global_ns() - t_begin < wait_limit_ns(abort_flag)) {
       }
     }
   } else if (warp >= 4 && n_iter > 0) {

@@ -285,7 +285,7 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
     }
     mbar_init(bars + 8 * kBbAll, 4 * kBWg);
     mbar_init(bars + 8 * kBbDrain, 1);
-    *abort_flag = 0;
+    wait_ctx_init(abort_flag, a.wait_limit_us);
     *grow_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -502,7 +502,7 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
     if (!ok) {
       umma_commit(bars + 8 * kBbDrain);
       const unsigned long long t_begin = global_ns();
-      while (!mbar_try_wait(bars + 8 * kBbDrain, 0) && global_ns() - t_begin < kWaitLimitNs) {
+      while (!mbar_try_wait(bars + 8 * kBbDrain, 0) && global_ns() - t_begin < wait_limit_ns(abort_flag)) {
       }
     }
   } else if (warp >= 4 && n_iter > 0) {

@@ -75,6 +75,9 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
                    int rows_pad, const TLayout lay) {
   constexpr int D = 128, HALVES = 2, KSTEPS_QK = D / 16;
   constexpr int CW = NP / 2;                        // rows (score columns) per softmax warpgroup
+  // the separate loop of plain tiles in the softmax warps: with 32 rows per warpgroup the second copy
+  // of the tile body pushes the register allocation into spills, which costs more than the walker
+  constexpr bool kPlainSoftmax = NP < 64;
   constexpr uint32_t kCols = NP <= 16 ? 64 : (NP <= 32 ? 128 : 256);   // S^T x2 and O^T, a power of two
   constexpr uint32_t kColO = 2 * NP;
   extern __shared__ __align__(1024) uint8_t smem[];
@@ -113,7 +116,7 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
     mbar_init(bars + 8 * kTbWg, 4);
     mbar_init(bars + 8 * (kTbWg + 1), 4);
     mbar_init(bars + 8 * kTbDrain, 1);
-    *abort_flag = 0;
+    wait_ctx_init(abort_flag, a.wait_limit_us);
     grow_flags[0] = 0;
     grow_flags[1] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -264,6 +267,53 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
     };
     ok = issue_qk();
     while (ok && wp.it < n_iter) {
+      // ---- a run of plain tiles needs neither walker.  S^T of a tile that neither opens nor closes
+      //      its piece is the same eight MMAs whatever the tile holds; O^T += V^T P^T of a full cache
+      //      tile that does not open its piece is eight accumulating MMAs.  Nearly every tile of a
+      //      long cache goes through this loop, whose only branches are the waits and the back edge.
+      if (wq.open && wp.open && wq.it == wp.it + 1) {
+        int n_run = min(min(wq.tiles_b - 1 - wq.ti, n_iter - 1 - wq.it), wp.L / kTile - wp.ti);
+        const uint32_t q_lo = q_lo0 + (wq.piece_idx & 1) * (lay.q_bytes >> 4);
+        int it = wp.it;
+        for (; n_run > 0; --n_run, ++it) {
+          // S^T(it + 1)
+          if (!mbar_wait(bars + 8 * (kTbKvFull + rk.buf), rk.par, abort_flag, status)) { ok = false; break; }
+          tc_fence_after();
+          {
+            const uint32_t k_lo = k_lo0 + rk.buf * (kKvBytes >> 4);
+            const uint32_t d_s = tmem + ((it + 1) & 1) * NP;
+#pragma unroll
+            for (int ks = 0; ks < KSTEPS_QK; ++ks)
+              umma_bf16_lo(d_s, k_lo + (ks >> 2) * (kHalfStrideT >> 4) + (ks & 3) * 2,
+                           q_lo + (ks >> 2) * (NP * 128 >> 4) + (ks & 3) * 2, idesc_qk, ks > 0);
+            umma_commit(bars + 8 * (kTbKvEmpty + rk.buf));
+            umma_commit(bars + 8 * (kTbSFull + ((it + 1) & 1)));
+            rk.step(2);
+          }
+          // O^T += V^T P^T (it)
+          if (!mbar_wait(bars + 8 * (kTbPFull + (it & 1)), (it >> 1) & 1, abort_flag, status) ||
+              !mbar_wait(bars + 8 * (kTbKvFull + rv.buf), rv.par, abort_flag, status)) {
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          {
+            const uint32_t p_lo = p_lo0 + (it & 1) * (kPBytes >> 4);
+            const uint32_t v_lo = v_lo0 + rv.buf * (kKvBytes >> 4);
+#pragma unroll
+            for (int j = 0; j < kTile / 16; ++j)
+              umma_bf16_lo(tmem + kColO, v_lo + j * (2048 >> 4), p_lo + j * (2048 >> 4), idesc_pv, 1u);
+            umma_commit(bars + 8 * (kTbKvEmpty + rv.buf));
+            umma_commit(bars + 8 * (kTbPvDone + (it & 1)));
+            rv.step(2);
+          }
+        }
+        if (!ok) break;
+        const int done = it - wp.it;
+        wq.ti += done; wq.it += done; wq.piece_j += done;
+        wp.ti += done; wp.it += done; wp.piece_j += done;
+        if (wp.it >= n_iter) break;
+      }
       // score buffer (it+1)&1 is free: the P^T of tile it-1 was waited for in the previous round
       if (wq.it < n_iter && !issue_qk()) { ok = false; break; }
       walk_tile(a, wp);
@@ -296,7 +346,7 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
       // aborting: let the tensor pipe run dry before tensor memory is released
       umma_commit(bars + 8 * kTbDrain);
       const unsigned long long t_begin = global_ns();
-      while (!mbar_try_wait(bars + 8 * kTbDrain, 0) && global_ns() - t_begin < kWaitLimitNs) {
+      while (!mbar_try_wait(bars + 8 * kTbDrain, 0) && global_ns() - t_begin < wait_limit_ns(abort_flag)) {
       }
     }
   } else if (warp >= 4 && n_iter > 0) {
@@ -328,83 +378,46 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
       ++wg_phase;
       return good;
     };
-    while (ok && w.it < n_iter) {
-      walk_tile(a, w);
-      const int it = w.it, pb = it & 1;
-      if (!wait_all(bars + 8 * (kTbSFull + pb), (it >> 1) & 1)) { ok = false; break; }
-      if (it >= 2 && !wait_all(bars + 8 * (kTbPvDone + pb), ((it >> 1) - 1) & 1)) { ok = false; break; }
-      tc_fence_after();
-      const int nv = w.nvalid;
-      if (w.is_step || nv < kTile) {
-        // V rows past the valid keys hold foreign or stale bytes; their P is 0 but 0 * NaN is NaN:
-        // clear the rows of the last 16-key step that the PV product still reads
-        const int use = 2 * it + 1, buf = use % lay.n_kv;
-        if (!wait_all(bars + 8 * (kTbKvFull + buf), (use / lay.n_kv) & 1)) { ok = false; break; }
-        const uint32_t va = sb + lay.off_kv + buf * kKvBytes;
-        const int n_rows = ((nv + 15) & ~15) - nv;
-        for (int x = wg * 128 + t; x < n_rows * HALVES * 8; x += 256) {
-          const int rr = nv + x / (HALVES * 8), cc = x % (HALVES * 8);
-          const uint32_t addr = va + (cc >> 3) * kHalfStrideT + rr * 128 + ((cc & 7) << 4);
-          asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(addr), "r"(0u) : "memory");
-        }
-      }
+    // scores of this key against the warpgroup's rows; invisible pairs become -inf
+    auto load_scores = [&](float (&v)[CW], uint32_t s_addr, int nv, bool is_step) {
+      uint32_t raw[CW];
+#pragma unroll
+      for (int c = 0; c < CW / 8; ++c) tmem_ld8(s_addr + c * 8, raw + c * 8);
+#pragma unroll
+      for (int c = 0; c < CW / 8; ++c) tmem_ld_wait8(raw + c * 8);
       const bool key_ok = t < nv;
-      const uint32_t s_addr = lane_addr + pb * NP + c0;
-
-      // scores of this key against the warpgroup's rows; invisible pairs become -inf
-      float v[CW];
-      auto load_scores = [&]() {
-        uint32_t raw[CW];
+      if (!is_step) {
 #pragma unroll
-        for (int c = 0; c < CW / 8; ++c) tmem_ld8(s_addr + c * 8, raw + c * 8);
-#pragma unroll
-        for (int c = 0; c < CW / 8; ++c) tmem_ld_wait8(raw + c * 8);
-        if (!w.is_step) {
-#pragma unroll
-          for (int j = 0; j < CW; ++j) v[j] = key_ok ? __uint_as_float(raw[j]) : -INFINITY;
-        } else {
-          int i = c0 / a.G, g = c0 - i * a.G;
-#pragma unroll
-          for (int j = 0; j < CW; ++j) {
-            bool vis = false;
-            if (key_ok && i < w.n_q) {
-              const int anc = (i < w.n_c) ? i : (a.anchor ? a.anchor[w.r0 + i] : w.n_c);
-              vis = step_key_visible(i, t, w.n_c, anc);
-            }
-            v[j] = vis ? __uint_as_float(raw[j]) : -INFINITY;
-            if (++g == a.G) { g = 0; ++i; }
-          }
-        }
-      };
-      // exact maximum over the tile's keys of every row -> red[warp][row]
-      auto reduce_row_max = [&]() {
-        float keep = -INFINITY;
+        for (int j = 0; j < CW; ++j) v[j] = key_ok ? __uint_as_float(raw[j]) : -INFINITY;
+      } else {
+        int i = c0 / a.G, g = c0 - i * a.G;
 #pragma unroll
         for (int j = 0; j < CW; ++j) {
-          const float r = warp_max_f32(v[j]);
-          if (lane == j) keep = r;
+          bool vis = false;
+          if (key_ok && i < w.n_q) {
+            const int anc = (i < w.n_c) ? i : (a.anchor ? a.anchor[w.r0 + i] : w.n_c);
+            vis = step_key_visible(i, t, w.n_c, anc);
+          }
+          v[j] = vis ? __uint_as_float(raw[j]) : -INFINITY;
+          if (++g == a.G) { g = 0; ++i; }
         }
-        red_w[lane] = keep;
-      };
-      auto red_max4 = [&](int j) -> float {
-        return fmaxf(fmaxf(red_g[j], red_g[32 + j]), fmaxf(red_g[64 + j], red_g[96 + j]));
-      };
-      load_scores();
-
-      if (w.piece_j == 0) {
-        // new unit: the reference maximum of each row is the exact maximum of this first tile
-        reduce_row_max();
-        if (!wg_sync()) { ok = false; break; }
-        if (t < CW) {
-          const float m = red_max4(t);
-          mref_g[t] = (m == -INFINITY) ? 0.f : m * a.scale_log2;
-        }
-        if (!wg_sync()) { ok = false; break; }
-#pragma unroll
-        for (int j = 0; j < CW; ++j) lsum[j] = 0.f;
       }
-
-      // x = s * scale - m_ref (log2 units)
+    };
+    // exact maximum over the tile's keys of every row -> red[warp][row]
+    auto reduce_row_max = [&](const float (&v)[CW]) {
+      float keep = -INFINITY;
+#pragma unroll
+      for (int j = 0; j < CW; ++j) {
+        const float r = warp_max_f32(v[j]);
+        if (lane == j) keep = r;
+      }
+      red_w[lane] = keep;
+    };
+    auto red_max4 = [&](int j) -> float {
+      return fmaxf(fmaxf(red_g[j], red_g[32 + j]), fmaxf(red_g[64 + j], red_g[96 + j]));
+    };
+    // x = s * scale - m_ref (log2 units); returns the largest x of this thread
+    auto shift_scores = [&](float (&v)[CW]) -> float {
       float tmaxx = -INFINITY;
 #pragma unroll
       for (int j4 = 0; j4 < CW / 4; ++j4) {
@@ -415,68 +428,149 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
         v[4 * j4 + 3] = fmaf(v[4 * j4 + 3], a.scale_log2, -m4.w);
         tmaxx = fmaxf(tmaxx, fmaxf(fmaxf(v[4 * j4], v[4 * j4 + 1]), fmaxf(v[4 * j4 + 2], v[4 * j4 + 3])));
       }
-      // the four warps agree on whether any score outgrew its reference (tile index as the token)
-      if (w.piece_j > 0 && __any_sync(0xffffffffu, tmaxx > kGrowLimit) && lane == 0) *grow_flag = it + 1;
-      if (!wg_sync()) { ok = false; break; }
-      if (*grow_flag == it + 1) {
-        // ---- rare: move the references up, rescale O^T and the partial sums, redo x ----
-        load_scores();
-        reduce_row_max();
-        if (!wg_sync()) { ok = false; break; }
-        float alpha[CW];
+      return tmaxx;
+    };
+    // ---- rare: move the references up, rescale O^T and the partial sums, redo x ----
+    auto regrow = [&](float (&v)[CW], int it, uint32_t s_addr, int nv, bool is_step) -> bool {
+      load_scores(v, s_addr, nv, is_step);
+      reduce_row_max(v);
+      if (!wg_sync()) return false;
+      float alpha[CW];
 #pragma unroll
-        for (int j = 0; j < CW; ++j) {
-          const float m = red_max4(j);
-          const float m_old = mref_g[j];
-          const float m_new = (m == -INFINITY) ? m_old : fmaxf(m_old, m * a.scale_log2);
-          alpha[j] = ex2(m_old - m_new);
-          lsum[j] *= alpha[j];
-          v[j] = fmaf(v[j], a.scale_log2, -m_new);
-        }
-        if (!wg_sync()) { ok = false; break; }          // everyone has read the old references
-        if (t < CW) {
-          const float m = red_max4(t);
-          if (m != -INFINITY) mref_g[t] = fmaxf(mref_g[t], m * a.scale_log2);
-        }
-        // all PV products issued so far are complete before O^T is touched
-        if (!wait_all(bars + 8 * (kTbPvDone + ((it - 1) & 1)), ((it - 1) >> 1) & 1)) { ok = false; break; }
-        tc_fence_after();
-        {
-          uint32_t o[CW];
-#pragma unroll
-          for (int c = 0; c < CW / 8; ++c) tmem_ld8(lane_addr + kColO + c0 + c * 8, o + c * 8);
-#pragma unroll
-          for (int c = 0; c < CW / 8; ++c) tmem_ld_wait8(o + c * 8);
-#pragma unroll
-          for (int j = 0; j < CW; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha[j]);
-#pragma unroll
-          for (int c = 0; c < CW / 8; ++c) tmem_st8(lane_addr + kColO + c0 + c * 8, o + c * 8);
-          asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-        }
-        if (!wg_sync()) { ok = false; break; }          // new references visible to later tiles
+      for (int j = 0; j < CW; ++j) {
+        const float m = red_max4(j);
+        const float m_old = mref_g[j];
+        const float m_new = (m == -INFINITY) ? m_old : fmaxf(m_old, m * a.scale_log2);
+        alpha[j] = ex2(m_old - m_new);
+        lsum[j] *= alpha[j];
+        v[j] = fmaf(v[j], a.scale_log2, -m_new);
       }
-
-      // p = 2^x as bf16 into this key's row of the P^T tile; partial row sums stay in registers
+      if (!wg_sync()) return false;          // everyone has read the old references
+      if (t < CW) {
+        const float m = red_max4(t);
+        if (m != -INFINITY) mref_g[t] = fmaxf(mref_g[t], m * a.scale_log2);
+      }
+      // all PV products issued so far are complete before O^T is touched
+      if (!wait_all(bars + 8 * (kTbPvDone + ((it - 1) & 1)), ((it - 1) >> 1) & 1)) return false;
+      tc_fence_after();
       {
-        const uint32_t p_row = sb + lay.off_p + pb * kPBytes + t * 128;
+        uint32_t o[CW];
 #pragma unroll
-        for (int c = 0; c < CW / 8; ++c) {
-          float p[8];
+        for (int c = 0; c < CW / 8; ++c) tmem_ld8(lane_addr + kColO + c0 + c * 8, o + c * 8);
 #pragma unroll
-          for (int e = 0; e < 8; ++e) {
-            p[e] = ex2(v[c * 8 + e]);
-            lsum[c * 8 + e] += p[e];
-          }
-          const uint32_t addr = p_row + (((c0 / 8 + c) ^ tx) << 4);
-          asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(pack2(p[0], p[1])),
-                       "r"(pack2(p[2], p[3])), "r"(pack2(p[4], p[5])), "r"(pack2(p[6], p[7]))
-                       : "memory");
-        }
+        for (int c = 0; c < CW / 8; ++c) tmem_ld_wait8(o + c * 8);
+#pragma unroll
+        for (int j = 0; j < CW; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha[j]);
+#pragma unroll
+        for (int c = 0; c < CW / 8; ++c) tmem_st8(lane_addr + kColO + c0 + c * 8, o + c * 8);
+        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
       }
+      return wg_sync();                      // new references visible to later tiles
+    };
+    // p = 2^x as bf16 into this key's row of the P^T tile; partial row sums stay in registers
+    auto emit_p = [&](const float (&v)[CW], int pb) {
+      const uint32_t p_row = sb + lay.off_p + pb * kPBytes + t * 128;
+#pragma unroll
+      for (int c = 0; c < CW / 8; ++c) {
+        float p[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          p[e] = ex2(v[c * 8 + e]);
+          lsum[c * 8 + e] += p[e];
+        }
+        const uint32_t addr = p_row + (((c0 / 8 + c) ^ tx) << 4);
+        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(pack2(p[0], p[1])),
+                     "r"(pack2(p[2], p[3])), "r"(pack2(p[4], p[5])), "r"(pack2(p[6], p[7]))
+                     : "memory");
+      }
+    };
+    // hands the P^T rows of this warp to the MMA thread
+    auto publish_p = [&](int pb) {
       fence_async_smem();
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bars + 8 * (kTbPFull + pb));
+    };
+    while (ok && w.it < n_iter) {
+      // ---- a run of plain tiles: full cache tiles that neither open nor close the piece need no
+      //      walker, no mask and none of the unit's begin / end work
+      if (kPlainSoftmax && w.open) {
+        int n_run = min(w.L / kTile - w.ti, n_iter - 1 - w.it);
+        for (; n_run > 0; --n_run) {
+          const int it = w.it, pb = it & 1;
+          // (the commit behind these scores also covers O^T += V^T P^T of tile it - 2: its P^T buffer is free)
+          if (!wait_all(bars + 8 * (kTbSFull + pb), (it >> 1) & 1)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t s_addr = lane_addr + pb * NP + c0;
+          float v[CW];
+          {
+            uint32_t raw[CW];
+#pragma unroll
+            for (int c = 0; c < CW / 8; ++c) tmem_ld8(s_addr + c * 8, raw + c * 8);
+#pragma unroll
+            for (int c = 0; c < CW / 8; ++c) tmem_ld_wait8(raw + c * 8);
+#pragma unroll
+            for (int j = 0; j < CW; ++j) v[j] = __uint_as_float(raw[j]);
+          }
+          const float tmaxx = shift_scores(v);
+          if (__any_sync(0xffffffffu, tmaxx > kGrowLimit) && lane == 0) *grow_flag = it + 1;
+          if (!wg_sync()) { ok = false; break; }
+          if (*grow_flag == it + 1 && !regrow(v, it, s_addr, kTile, false)) { ok = false; break; }
+          emit_p(v, pb);
+          publish_p(pb);
+          ++w.ti;
+          ++w.it;
+          ++w.piece_j;
+        }
+        if (!ok) break;
+      }
+      walk_tile(a, w);
+      const int it = w.it, pb = it & 1;
+      if (!wait_all(bars + 8 * (kTbSFull + pb), (it >> 1) & 1)) { ok = false; break; }
+      tc_fence_after();
+      const int nv = w.nvalid;
+      const uint32_t s_addr = lane_addr + pb * NP + c0;
+      float v[CW];
+      load_scores(v, s_addr, nv, w.is_step);
+
+      if (w.piece_j == 0) {
+        // new unit: the reference maximum of each row is the exact maximum of this first tile
+        reduce_row_max(v);
+        if (!wg_sync()) { ok = false; break; }
+        if (t < CW) {
+          const float m = red_max4(t);
+          mref_g[t] = (m == -INFINITY) ? 0.f : m * a.scale_log2;
+        }
+        if (!wg_sync()) { ok = false; break; }
+#pragma unroll
+        for (int j = 0; j < CW; ++j) lsum[j] = 0.f;
+      }
+
+      const float tmaxx = shift_scores(v);
+      if (w.piece_j > 0) {
+        // the four warps agree on whether any score outgrew its reference (tile index as the token);
+        // a piece's first tile set the references from its own scores and cannot outgrow them
+        if (__any_sync(0xffffffffu, tmaxx > kGrowLimit) && lane == 0) *grow_flag = it + 1;
+        if (!wg_sync()) { ok = false; break; }
+        if (*grow_flag == it + 1 && !regrow(v, it, s_addr, nv, w.is_step)) { ok = false; break; }
+      }
+      emit_p(v, pb);
+      if (w.is_step || nv < kTile) {
+        // V rows past the valid keys hold foreign or stale bytes; their P is 0 but 0 * NaN is NaN:
+        // clear the rows of the last 16-key step that the PV product still reads.  Done behind the
+        // exponentials, so that the wait for the V tile (which lands after the K tile) overlaps them,
+        // and before P^T is handed over, so that the product sees the cleared rows.
+        const int use = 2 * it + 1, buf = use % lay.n_kv;
+        if (!wait_all(bars + 8 * (kTbKvFull + buf), (use / lay.n_kv) & 1)) { ok = false; break; }
+        const uint32_t va = sb + lay.off_kv + buf * kKvBytes;
+        const int n_rows = ((nv + 15) & ~15) - nv;
+        for (int x = wg * 128 + t; x < n_rows * HALVES * 8; x += 256) {
+          const int rr = nv + x / (HALVES * 8), cc = x % (HALVES * 8);
+          const uint32_t addr = va + (cc >> 3) * kHalfStrideT + rr * 128 + ((cc & 7) << 4);
+          asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(addr), "r"(0u) : "memory");
+        }
+      }
+      publish_p(pb);
 
       if (w.last) {
         // ---- end of the unit (or of this CTA's part of it) ----
@@ -505,15 +599,17 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
         __nv_bfloat16* out_l = a.out + w.layer * a.out_layer_stride;
         float* lse_l = a.lse ? a.lse + w.layer * a.lse_layer_stride : nullptr;
         if (w.slot < 0) {
-          int i = c0 / a.G, g = c0 - i * a.G;
+          const int i0 = c0 / a.G;
+          int g = c0 - i0 * a.G;
+          int64_t orow = static_cast<int64_t>(w.r0 + i0) * a.H_q + w.h * a.G + g;
+          const int64_t next_token = a.H_q - a.G + 1;      // from the last head of a token's group to the first of the next
 #pragma unroll
           for (int j = 0; j < CW; ++j) {
             if (c0 + j < rows) {
-              const int64_t orow = static_cast<int64_t>(w.r0 + i) * a.H_q + w.h * a.G + g;
-              out_l[orow * D + t] = __float2bfloat16_rn(__uint_as_float(o[j]) / l_row[j]);
+              out_l[orow * D + t] = __float2bfloat16_rn(__uint_as_float(o[j]) * __frcp_rn(l_row[j]));
               if (lse_l && t == j) lse_l[orow] = (m_mine + log2f(l_row[j])) * 0.69314718055994531f;
             }
-            if (++g == a.G) { g = 0; ++i; }
+            if (++g == a.G) { g = 0; orow += next_token; } else { ++orow; }
           }
         } else {
           float* slot = ws_slots + static_cast<size_t>(w.slot) * ws_slot_floats(D, rows_pad);
@@ -620,8 +716,13 @@ int32_t launch_attn_umma_t(const AttnArgs& a_in, cudaStream_t st) {
   if (static_cast<int>((a.B + 1 + kTThreads / 32) * sizeof(int)) > lay.n_kv * kKvBytes) return MS_ERR_UNSUPPORTED_SHAPE;
   const int grid = attn_mma_grid();
   if (grid <= 0) return cuda_status(cudaErrorNoDevice);
-  // the merge runs in the kernel's tail when a bank of counters is to be had (two per CTA)
-  a.done = (2 * grid <= kDoneBankWords) ? done_bank(a.workspace) : nullptr;
+  // Where the merge runs.  With at least two units per CTA a unit is cut into two or three pieces
+  // and the warpgroup that delivers the last of them merges it on the spot (counters: two per
+  // CTA).  With few units -- a small batch -- every unit is cut across many CTAs, and merging a
+  // unit inside one CTA would leave the rest of the machine idle meanwhile: the merge is then a
+  // launch of its own, one warp per (unit, row), behind this kernel.
+  const long long units = static_cast<long long>(a.n_layers) * a.B * a.H_kv;
+  a.done = (units >= 2ll * grid && 2 * grid <= kDoneBankWords) ? done_bank(a.workspace) : nullptr;
   // one descriptor per tensor covers every layer (the layer is the outermost coordinate)
   const uint64_t nl = static_cast<uint64_t>(a.n_layers);
   const uint64_t kv_ls = nl > 1 ? a.kv_layer_stride : static_cast<uint64_t>(a.H_kv) * a.kv_head_stride;

@@ -34,6 +34,9 @@ int32_t sm_count();
 
 inline cudaStream_t as_stream(memosight_stream_t s) { return reinterpret_cast<cudaStream_t>(s); }
 
+// Limit of one bounded device-side wait, in microseconds (memosight_debug_set_wait_limit_us).
+unsigned int wait_limit_us();
+
 // "Last block done" counters (done_banks.cu): the zero-initialised bank of kDoneBankWords
 // counters that belongs to `key` on the current device, or nullptr when every bank is taken
 // (the caller then uses its two-launch form).  A kernel must leave its counters at zero.

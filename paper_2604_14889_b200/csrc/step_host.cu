@@ -1,4 +1,4 @@
-// One whole decode step driven from host-resident step data: copies in, the
+// One whole decode step, by default driven from host-resident step data: copies in, the
 // kernels of the hot path in their order (Algorithm 1: forward pass attention,
 // greedy accept, S <- S (+) A, optional UpdateCache), copies out.  Pure
 // sequencing of the other entry points on the caller's stream -- except that the
@@ -50,31 +50,35 @@ extern "C" int32_t memosight_step_host(const memosight_step_host_params* p,
   if (T < 0 || B < 0 || a.n_q_heads < 1 || a.n_kv_heads < 1 || a.head_dim < 1 || p->vocab < 0)
     return MS_ERR_INVALID_ARG;
   if (T == 0 || B == 0) return MS_OK;
-  if (!p->h_q || !p->h_k_step || !p->h_v_step || !p->h_pos_id || !p->d_pos_id || !p->h_out || !a.q ||
-      !a.k_step || !a.v_step || !a.out)
-    return MS_ERR_INVALID_ARG;
-  if (p->vocab > 0 && (!p->h_logits || !p->d_logits || !p->h_draft || !p->d_draft || !p->d_argmax ||
-                       !p->d_n_match || !p->d_n_keep || p->ld_v < p->vocab))
+  if (!p->d_pos_id || !a.q || !a.k_step || !a.v_step || !a.out) return MS_ERR_INVALID_ARG;
+  if (p->vocab > 0 && (!p->d_logits || !p->d_draft || !p->d_argmax || !p->d_n_match || !p->d_n_keep ||
+                       p->ld_v < p->vocab))
     return MS_ERR_INVALID_ARG;
   cudaStream_t st = ms::as_stream(stream);
   const size_t q_bytes = static_cast<size_t>(T) * a.n_q_heads * a.head_dim * 2;
   const size_t kv_bytes = static_cast<size_t>(T) * a.n_kv_heads * a.head_dim * 2;
   // ---- host -> device: the step's inputs
-  MS_CUDA_TRY(cudaMemcpyAsync(const_cast<void*>(a.q), p->h_q, q_bytes, cudaMemcpyHostToDevice, st));
-  MS_CUDA_TRY(cudaMemcpyAsync(const_cast<void*>(a.k_step), p->h_k_step, kv_bytes, cudaMemcpyHostToDevice, st));
-  MS_CUDA_TRY(cudaMemcpyAsync(const_cast<void*>(a.v_step), p->h_v_step, kv_bytes, cudaMemcpyHostToDevice, st));
-  MS_CUDA_TRY(cudaMemcpyAsync(p->d_pos_id, p->h_pos_id, sizeof(int32_t) * T, cudaMemcpyHostToDevice, st));
+  if (p->h_q) MS_CUDA_TRY(cudaMemcpyAsync(const_cast<void*>(a.q), p->h_q, q_bytes, cudaMemcpyHostToDevice, st));
+  if (p->h_k_step)
+    MS_CUDA_TRY(cudaMemcpyAsync(const_cast<void*>(a.k_step), p->h_k_step, kv_bytes, cudaMemcpyHostToDevice, st));
+  if (p->h_v_step)
+    MS_CUDA_TRY(cudaMemcpyAsync(const_cast<void*>(a.v_step), p->h_v_step, kv_bytes, cudaMemcpyHostToDevice, st));
+  if (p->h_pos_id)
+    MS_CUDA_TRY(cudaMemcpyAsync(p->d_pos_id, p->h_pos_id, sizeof(int32_t) * T, cudaMemcpyHostToDevice, st));
   CopyLane* lane = nullptr;
-  if (p->vocab > 0) {
+  const bool side_copy = p->vocab > 0 && (p->h_logits || p->h_draft);
+  if (side_copy) {
     // the logits go their own way: behind whatever `stream` holds now (the previous step's accept
     // may still read the staging buffer), beside RoPE and the attention, back in before the accept
     const int32_t rc_lane = copy_lane(&lane);
     if (rc_lane != MS_OK) return rc_lane;
     MS_CUDA_TRY(cudaEventRecord(lane->fork, st));
     MS_CUDA_TRY(cudaStreamWaitEvent(lane->stream, lane->fork, 0));
-    MS_CUDA_TRY(cudaMemcpyAsync(p->d_logits, p->h_logits, sizeof(float) * static_cast<size_t>(T) * p->ld_v,
-                                cudaMemcpyHostToDevice, lane->stream));
-    MS_CUDA_TRY(cudaMemcpyAsync(p->d_draft, p->h_draft, sizeof(int32_t) * T, cudaMemcpyHostToDevice, lane->stream));
+    if (p->h_logits)
+      MS_CUDA_TRY(cudaMemcpyAsync(p->d_logits, p->h_logits, sizeof(float) * static_cast<size_t>(T) * p->ld_v,
+                                  cudaMemcpyHostToDevice, lane->stream));
+    if (p->h_draft)
+      MS_CUDA_TRY(cudaMemcpyAsync(p->d_draft, p->h_draft, sizeof(int32_t) * T, cudaMemcpyHostToDevice, lane->stream));
     MS_CUDA_TRY(cudaEventRecord(lane->join, lane->stream));
   }
   // ---- the hot path
@@ -85,7 +89,7 @@ extern "C" int32_t memosight_step_host(const memosight_step_host_params* p,
   rc = memosight_attn_step(&a, stream);
   if (rc != MS_OK) return rc;
   if (p->vocab > 0) {
-    MS_CUDA_TRY(cudaStreamWaitEvent(st, lane->join, 0));
+    if (side_copy) MS_CUDA_TRY(cudaStreamWaitEvent(st, lane->join, 0));
     rc = memosight_accept(p->d_logits, p->ld_v, p->vocab, a.q_off, B, T, p->d_draft, p->d_argmax,
                           p->d_n_match, p->d_n_keep, p->accept_workspace, p->accept_workspace_bytes,
                           stream);
@@ -105,7 +109,7 @@ extern "C" int32_t memosight_step_host(const memosight_step_host_params* p,
     if (rc != MS_OK) return rc;
   }
   // ---- device -> host: the step's results
-  MS_CUDA_TRY(cudaMemcpyAsync(p->h_out, a.out, q_bytes, cudaMemcpyDeviceToHost, st));
+  if (p->h_out) MS_CUDA_TRY(cudaMemcpyAsync(p->h_out, a.out, q_bytes, cudaMemcpyDeviceToHost, st));
   if (p->vocab > 0) {
     if (p->h_argmax)
       MS_CUDA_TRY(cudaMemcpyAsync(p->h_argmax, p->d_argmax, sizeof(int32_t) * T, cudaMemcpyDeviceToHost, st));

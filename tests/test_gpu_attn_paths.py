@@ -154,3 +154,26 @@ def test_forced_rows_path_never_outgrows_the_workspace(force_path, G, nq):
     want, want_lse = oracle_attn(P)
     out, lse = gpu_attn(P, ws_min_bytes=64 << 20)
     assert_attn_close(out, lse, want, want_lse, f"forced rows-on-lanes, large workspace G={G} nq={nq}")
+
+
+def test_a_wait_that_runs_out_is_reported_and_leaves_the_device_usable():
+    # The failure path of the bounded waits, without anything failing: one warp waits 3 ms on a
+    # barrier at which nobody arrives; the wait gives up, the kernel returns, the status word says so
+    # once, and the next attention call on the same workspace is served as usual.
+    P = random_problem(2, 8, 2, 128, [300, 40], [6, 6], [3, 3], seed=2)
+    ws_bytes = ms.memosight_attn_workspace_bytes(2, 8, 2, 128, 300, 6)
+    ws = torch.zeros(ws_bytes, dtype=torch.uint8, device="cuda")
+    assert ms.memosight_attn_status(ws) == ms.MS_OK
+    ms.memosight_debug_wait_timeout(ws, 3000)
+    assert ms.memosight_attn_status(ws) == ms.MS_ERR_DEVICE_TIMEOUT
+    assert ms.memosight_attn_status(ws) == ms.MS_OK              # reported once, then cleared
+    with pytest.raises(ms.MemosightError):
+        ms.memosight_debug_wait_timeout(ws, 5_000_000)           # limits beyond a second are refused
+    # the limit of the real kernels is a launch parameter too
+    prev = ms.memosight_debug_set_wait_limit_us(2_000_000)
+    try:
+        assert ms.memosight_debug_set_wait_limit_us(0) == 2_000_000
+        check_attn(P, "after a timed-out wait")
+    finally:
+        ms.memosight_debug_set_wait_limit_us(prev)
+    assert ms.memosight_debug_set_wait_limit_us(0) == prev
