@@ -140,7 +140,7 @@ class ClockSampler(threading.Thread):
 
     def __init__(self, index):
         super().__init__(daemon=True)
-        self.index, self.samples, self.reasons, self.max_mhz = index, [], set(), None
+        self.index, self.samples, self.times, self.reasons, self.max_mhz = index, [], [], set(), None
         self._stop_evt = threading.Event()
         self.ok = False
         try:
@@ -166,6 +166,7 @@ class ClockSampler(threading.Thread):
         while not self._stop_evt.is_set():
             try:
                 self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                self.times.append(time.perf_counter())
                 mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
                 for k, bit in names.items():
                     if mask & bit:
@@ -390,7 +391,7 @@ def main():
     if args.graph and n_e2e:
         raise SystemExit("--graph needs --no-e2e")
     n_sched = n_total + (3 + n_e2e if n_e2e else 0) + (2 * K + 1 if args.graph else 0)
-    growth = 3 * n_sched + SEG_LEN + 64
+    growth = max(3, cfg0.n_cand) * n_sched + SEG_LEN + 64
     cfg = synth.StepConfig(cfg0.name, cfg0.batch, cfg0.n_q_heads, cfg0.n_kv_heads, cfg0.head_dim, cfg0.len_lo,
                            cfg0.len_hi, cfg0.n_cand, cfg0.d, cfg0.rope_base, cfg0.vocab, headroom=growth,
                            seed=cfg0.seed + 1000 * rank)
@@ -455,11 +456,13 @@ def main():
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     sampler.start()
+    t_wall0 = time.perf_counter()
     e0.record()
     for s in range(K):
         step(W + s, ev_pairs[s])
     e1.record()
     barrier()
+    t_wall1 = time.perf_counter()
     clocks = sampler.finish()
     elapsed_ms = e0.elapsed_time(e1)
     split_ms = [a_.elapsed_time(b_) for a_, b_ in ev_pairs]
@@ -545,6 +548,25 @@ def main():
                 "traffic": None if NCU_TRAFFIC_PER_ALGO_BYTE is None else NCU_TRAFFIC_PER_ALGO_BYTE * algo_per_launch,
                 "share_of_step_time": split_avg_ms * K / elapsed_ms}
 
+    # a long run: the attention kernel's time binned by the SM clock that was sampled while it ran
+    sustained = None
+    if elapsed_ms >= 1000.0 and len(sampler.samples) >= 20:
+        ts, mhz = np.array(sampler.times), np.array(sampler.samples, dtype=float)
+        # steps are issued back to back and the device is the bottleneck: step i ran at about this wall time
+        step_t = t_wall1 - (elapsed_ms * 1e-3) * (1.0 - (np.arange(K) + 0.5) / K)
+        step_mhz = mhz[np.clip(np.searchsorted(ts, step_t), 0, len(mhz) - 1)]
+        bins = []
+        for c in sorted(set(step_mhz.tolist())):
+            sel = step_mhz == c
+            ms_c = float(np.mean(np.array(split_ms)[sel]))
+            by_c = float(np.mean(np.array(kv_bytes)[sel])) + step_local
+            bins.append({"sm_mhz": c, "steps": int(sel.sum()), "attn_ms": ms_c, "gbs": by_c / (ms_c * 1e-3) / 1e9,
+                         "attn_ms_x_ghz": ms_c * c / 1000.0})
+        sustained = {"timed_seconds": elapsed_ms / 1e3, "median_sm_mhz": float(np.median(mhz)),
+                     "attn_ms_x_median_ghz": split_avg_ms * float(np.median(mhz)) / 1000.0, "by_clock": bins,
+                     "note": "per-step time of the split-KV kernel grouped by the SM clock sampled nearest to the step "
+                             "(NVML, every 20 ms); a bandwidth that does not follow the clock is HBM-bound"}
+
     # ---- end to end: the step's inputs and results live in pinned host memory
     e2e = None
     if not args.no_e2e:
@@ -570,6 +592,8 @@ def main():
         line["graph"] = graph_info
     if one_call is not None:
         line["one_call"] = one_call
+    if sustained is not None:
+        line["sustained"] = sustained
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
             del inp, acc
@@ -680,7 +704,7 @@ def run_config(args, ms, dev):
     B, Hq, Hkv, D, nq = cfg0.batch, cfg0.n_q_heads, cfg0.n_kv_heads, cfg0.head_dim, cfg0.n_q
     T = B * nq
     lens0 = synth.make_lengths(cfg0)
-    n_rounds = 4                                    # whole, graph, parts, per-layer (or L2-warm)
+    n_rounds = 5                                    # whole, graph, parts, split kernel, per-layer (or L2-warm)
     growth = cfg0.n_cand * (W + K + 2) * (n_rounds + 1) + 64
     if name == "longcot":
         growth = max(growth, SEG_LEN + MEM_TOKENS + 64)
@@ -858,18 +882,28 @@ def run_config(args, ms, dev):
         for a_, b_ in row:
             a_.record()
             b_.record()
-    kv_parts = kv_bytes_mean(K)
     for s_ in range(K):
         m = marks[s_]
         m[0].record()
         rope()
         m[1].record()
-        attn(True, ev=evs[s_] if NL > 1 else evs[s_][0])
+        attn(True)
         m[2].record()
         accept()
         m[3].record()
         append()
         m[4].record()
+        state["step"] += 1
+    torch.cuda.synchronize()
+    advance(K)
+    # ---- round 2b: the split-KV kernel alone (events recorded by the library right around it; no other
+    #      event in the step, so that nothing but the kernel lies between the two)
+    kv_parts = kv_bytes_mean(K)
+    for s_ in range(K):
+        rope()
+        attn(True, ev=evs[s_] if NL > 1 else evs[s_][0])
+        accept()
+        append()
         state["step"] += 1
     torch.cuda.synchronize()
     advance(K)

@@ -15,7 +15,7 @@ constexpr int kMaxE = 8;   // D <= 256
 
 __global__ void __launch_bounds__(kWarps * 32)
 attn_simt_kernel(AttnArgs a) {
-  const int hq = blockIdx.x, t = blockIdx.y;
+  const int t = blockIdx.x, hq = blockIdx.y;       // rows on grid.x: no 65535 limit on the block rows
   const int D = a.D, E = D >> 5;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   // sequence of this row: largest b with q_off[b] <= t
@@ -25,11 +25,17 @@ attn_simt_kernel(AttnArgs a) {
     if (a.q_off[mid] <= t) lo = mid; else hi = mid;
   }
   const int b = lo;
-  const int r0 = a.q_off[b], n_q = a.q_off[b + 1] - r0;
+  // block size and cache length are clamped to the host's bounds, as on the tensor-core paths
+  const int r0 = a.q_off[b];
+  int n_q = a.q_off[b + 1] - r0;
+  n_q = n_q < 0 ? 0 : (n_q > a.max_nq ? a.max_nq : n_q);
   if (t < r0 || t >= r0 + n_q) return;
-  const int i = t - r0, n_c = a.n_cand[b];
+  int n_c = a.n_cand[b];
+  n_c = n_c < 0 ? 0 : (n_c > n_q ? n_q : n_c);
+  const int i = t - r0;
   const int a_i = (i < n_c) ? i : (a.anchor ? a.anchor[t] : n_c);
-  const int L = a.kv_len[b];
+  int L = a.kv_len[b];
+  L = L < 0 ? 0 : (L > a.max_kv_len ? a.max_kv_len : L);
   const int kvh = hq / a.G;
   const __nv_bfloat16* Kc = a.k_cache + kvh * a.kv_head_stride + a.kv_off[b] * static_cast<int64_t>(D);
   const __nv_bfloat16* Vc = a.v_cache + kvh * a.kv_head_stride + a.kv_off[b] * static_cast<int64_t>(D);
@@ -92,8 +98,7 @@ attn_simt_kernel(AttnArgs a) {
 
 int32_t launch_attn_simt(const AttnArgs& a, cudaStream_t st) {
   if (a.T == 0) return MS_OK;
-  if (a.T > 65535) return MS_ERR_UNSUPPORTED_SHAPE;
-  attn_simt_kernel<<<dim3(a.H_q, a.T), kWarps * 32, 0, st>>>(a);
+  attn_simt_kernel<<<dim3(a.T, a.H_q), kWarps * 32, 0, st>>>(a);
   MS_LAUNCH_CHECK();
   return MS_OK;
 }

@@ -513,6 +513,7 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
     const uint32_t rx = r & 7;
     BigWalk w = w0;
     float m_ref = 0.f, l_part = 0.f;
+    bool unref = false;     // the row has not seen a visible key in this item yet: it has no reference
     int tok = 0, anc = 0, rows = 0;
     bool row_ok = false;
     uint32_t all_phase = 0;
@@ -580,7 +581,13 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
         s_mx[wg * kTile + r] = max_cols(v);
         if (!sync_all()) return false;
         const float m = max_of_groups(s_mx);
-        m_ref = (m == -INFINITY) ? 0.f : m * a.scale_log2;
+        // A row that sees no key in the item's first tile (a chunk that starts right of the row's
+        // causal limit, a foresight row with anchor 0, a training-mask row behind other steps' tokens)
+        // stays without a reference: the first later tile with a visible key sets it through the
+        // branch below, whatever the size of its scores (a placeholder of 0 would flush strongly
+        // negative rows to a zero sum).
+        unref = (m == -INFINITY);
+        m_ref = unref ? 0.f : m * a.scale_log2;
         l_part = 0.f;
       }
       // p = 2^(s*scale - m_ref) as bf16 into this row of the P tile; the row's partial sum over
@@ -588,35 +595,46 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
       const uint32_t p_row = sb + kBOffP + pb * kBPBytes + ((wg * kBCw) >> 6) * kBHalf + r * 128;
       const int chunk0 = ((wg * kBCw) & 63) >> 3;             // first 16-byte chunk inside the 64-key half
       auto p_pass = [&]() -> float {
-        float ls[4] = {0.f, 0.f, 0.f, 0.f};
+        // scale-and-shift and the running sums two values per instruction (packed fp32 pairs)
+        const f32x2_t scale2 = pack_f32x2(a.scale_log2, a.scale_log2), nm2 = pack_f32x2(-m_ref, -m_ref);
+        f32x2_t ls[2] = {pack_f32x2(0.f, 0.f), pack_f32x2(0.f, 0.f)};
   #pragma unroll
         for (int c = 0; c < kBCw / 8; ++c) {
           float p[8];
   #pragma unroll
-          for (int e = 0; e < 8; ++e) {
-            p[e] = ex2(fmaf(v[c * 8 + e], a.scale_log2, -m_ref));
-            ls[e & 3] += p[e];
+          for (int e = 0; e < 8; e += 2) {
+            float x0, x1;
+            unpack_f32x2(fma_f32x2(pack_f32x2(v[c * 8 + e], v[c * 8 + e + 1]), scale2, nm2), x0, x1);
+            p[e] = ex2(x0);
+            p[e + 1] = ex2(x1);
+            ls[(e >> 1) & 1] = add_f32x2(ls[(e >> 1) & 1], pack_f32x2(p[e], p[e + 1]));
           }
           const uint32_t addr = p_row + (((chunk0 + c) ^ rx) << 4);
           asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(pack2(p[0], p[1])),
                        "r"(pack2(p[2], p[3])), "r"(pack2(p[4], p[5])), "r"(pack2(p[6], p[7]))
                        : "memory");
         }
-        return (ls[0] + ls[1]) + (ls[2] + ls[3]);
+        float s0, s1, s2, s3;
+        unpack_f32x2(ls[0], s0, s1);
+        unpack_f32x2(ls[1], s2, s3);
+        return (s0 + s1) + (s2 + s3);
       };
       float tsum = p_pass();
       // A score that outgrew the row reference by ~2^48 shows in the sum (so do inf and NaN); the
       // softmax warps agree on it before anyone hands P over
-      if (!opens_item && __any_sync(0xffffffffu, row_ok && !(tsum < kBGrowSum)) && lane == 0)
-        *grow_flag = it + 1;
+      bool regrow = row_ok && !(tsum < kBGrowSum);
+      if (unref && row_ok) regrow = max_cols(v) > -INFINITY;       // the row's first visible key: set its reference
+      if (!opens_item && __any_sync(0xffffffffu, regrow) && lane == 0) *grow_flag = it + 1;
       if (!sync_all()) return false;
       if (*grow_flag == it + 1) {
         // ---- rare: move the row references up; rescale O (this group's columns) and the sums ----
         s_mx[wg * kTile + r] = max_cols(v);
         if (!sync_all()) return false;
         const float m = max_of_groups(s_mx);
-        const float m_new = (m == -INFINITY) ? m_ref : fmaxf(m_ref, m * a.scale_log2);
-        const float alpha = ex2(m_ref - m_new);
+        const float m_new = (m == -INFINITY) ? m_ref : (unref ? m * a.scale_log2 : fmaxf(m_ref, m * a.scale_log2));
+        // (a row without a reference has accumulated nothing: its O and sum are zero and stay so)
+        const float alpha = unref ? 1.f : ex2(m_ref - m_new);
+        if (m != -INFINITY) unref = false;
         m_ref = m_new;
         l_part *= alpha;
         if (!wait_all(bar_pv_done(it - 1), ((it - 1) >> 1) & 1)) return false;

@@ -103,3 +103,23 @@ def test_long_blocks_whose_key_tiles_left_of_the_diagonal_still_need_the_mask():
     check_attn(random_problem(2, 8, 2, 128, [129, 0], [400, 300], [350, 260], seed=54, anchors=True),
                "long blocks with custom anchors")
     check_attn(random_problem(1, 4, 1, 128, [0], [640], [640], seed=55), "all candidates, G = 4, one head")
+
+
+def test_rows_that_see_nothing_at_first_and_only_strongly_negative_scores_later():
+    # Foresight rows with anchor 0 see themselves only.  In a long block with an empty cache such a
+    # row finds no visible key in its item's first key tile; its one key comes tiles later -- and here
+    # it scores 150 nats below zero, far beyond what an exponential against a placeholder reference
+    # of 0 can represent.  The softmax over that single key is still exactly its V row.
+    P = random_problem(1, 8, 2, 128, [0], [300], [120], seed=61, anchors=True)
+    rows = [130, 201, 299]                       # foresight rows in the second and third key tile
+    for i in rows:
+        P["anchor"][i] = 0
+        for kvh in range(2):
+            q = P["q"][i, kvh * 4].float()      # first query head of the group: its score on key i is -150
+            P["k_step"][i, kvh] = (-150.0 * np.sqrt(128) * q / q.norm() ** 2).to(torch.bfloat16)
+    out, lse = check_attn(P, "unreferenced rows, strongly negative scores")
+    for i in rows:
+        for kvh in range(2):
+            assert torch.equal(out[i, kvh * 4], P["v_step"][i, kvh]), "a single visible key: the output is its V row"
+            assert abs(float(lse[i, kvh * 4]) + 150.0) < 1.0
+    assert bool(torch.isfinite(out.float()).all())

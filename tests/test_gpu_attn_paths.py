@@ -177,3 +177,20 @@ def test_a_wait_that_runs_out_is_reported_and_leaves_the_device_usable():
     finally:
         ms.memosight_debug_set_wait_limit_us(prev)
     assert ms.memosight_debug_set_wait_limit_us(0) == prev
+
+
+def test_general_path_many_rows_and_clamped_lengths(force_path):
+    # more than 65535 block rows in one call (head_dim 32 only has the general kernel)
+    B, nq = 4200, 16
+    lens = [(3 * b) % 7 for b in range(B)]
+    P = random_problem(B, 2, 1, 32, lens, [nq] * B, [(b % (nq + 1)) for b in range(B)], seed=88, headroom=1)
+    assert P["T"] > 65535
+    check_attn(P, "general path, 67200 rows")
+    # a device length above the host's bound is clamped to the bound, on this path as on the others:
+    # the result is that of a cache of max_kv_len entries
+    force_path("general")
+    Q = random_problem(3, 8, 2, 128, [300, 40, 129], [6, 6, 6], [3, 3, 3], seed=89, headroom=64)
+    want, want_lse = oracle_attn(Q)
+    # (the harness passes max(lens) = 300 as max_kv_len and the tensor below as the device lengths)
+    out, lse = gpu_attn(dict(Q, kv_len=torch.tensor([300 + 40, 40, 129], dtype=torch.int32)))
+    assert_attn_close(out, lse, want, want_lse, "kv_len above max_kv_len is clamped")

@@ -130,3 +130,44 @@ def test_output_budget_ends_a_sequence():
     seqs, _ = run_oracle_loop(m, _params(m, 3, max_out=10), [0], [0], max_steps=50)
     assert len(seqs[0].out) == 10 and (seqs[0].flags & od.DONE)
     assert seqs[0].out == plain_greedy(m, 0, 0, 10)
+
+
+def test_compression_block_is_forwarded_before_the_eviction():
+    # The reading this repository takes of Algorithm 1 (Forward of <m_1..m_l, o>, then UpdateCache):
+    # the whole compression block -- <o> included -- is one causal block forwarded while the finished
+    # step's verbose entries are still in the cache, so every row of it attends to them (Sec. 2.3
+    # names reasoning and memory tokens as attending to the current step; <o> follows the memory
+    # tokens in the same forward pass and is given the same view).  Pinned here: perturbing one
+    # verbose entry changes the memory tokens' AND <o>'s output; after the eviction a later block no
+    # longer sees that entry.
+    from conftest import bits, from_bits
+    import torch
+    g = torch.Generator().manual_seed(3)
+    D, n, l = 32, 6, 2                                    # a 6-token step, two memory tokens + <o>
+    L0 = 5                                                # prompt entries in front of the step
+    rnd = lambda *s: torch.randn(s, generator=g).to(torch.bfloat16)
+    k_cache, v_cache = rnd(1, 32, D), rnd(1, 32, D)
+    q, ks, vs = rnd(l + 1, 1, D), rnd(l + 1, 1, D), rnd(l + 1, 1, D)
+    kv_off, kv_len = np.array([0], np.int64), np.array([L0 + n], np.int32)
+    q_off, n_cand = np.array([0, l + 1], np.int32), np.array([l + 1], np.int32)
+
+    def forward(kc):
+        out, _ = oracle.attn_step(bits(kc), bits(v_cache), 32 * D, kv_off, kv_len, q_off, n_cand, None, bits(q), bits(ks),
+                                  bits(vs))
+        return out
+    base = forward(k_cache)
+    k2 = k_cache.clone()
+    k2[0, L0 + 2] = rnd(D) * 4                            # one verbose entry of the finished step
+    moved = forward(k2)
+    for row in range(l + 1):                              # both <m> rows and the <o> row see it
+        assert np.abs(moved[row] - base[row]).max() > 1e-3
+    # after UpdateCache the entry is gone for everybody that comes later
+    kb, vb, len2 = bits(k2), bits(v_cache), kv_len.copy()
+    oracle.kv_append(kb[0], vb[0], 32 * D, 1, D, kv_off, len2, bits(ks), bits(vs), q_off, n_cand, np.array([l + 1]))
+    oracle.kv_compact(kb, vb, 1, 32 * D, 32 * D, 1, D, kv_off, len2, [L0], [n])
+    assert len2.tolist() == [L0 + l + 1]
+    kb0 = bits(k_cache)
+    len0 = kv_len.copy()
+    oracle.kv_append(kb0[0], vb[0].copy(), 32 * D, 1, D, kv_off, len0, bits(ks), bits(vs), q_off, n_cand, np.array([l + 1]))
+    oracle.kv_compact(kb0, vb.copy(), 1, 32 * D, 32 * D, 1, D, kv_off, len0, [L0], [n])
+    assert np.array_equal(kb[0][0, :L0 + l + 1], kb0[0][0, :L0 + l + 1])
