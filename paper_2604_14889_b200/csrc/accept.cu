@@ -10,9 +10,10 @@
 // the ring and reduce it with shuffles only.  Other layouts fall back to one CTA per
 // (chunk, row) with plain loads.  Pass 2 folds the chunk candidates of every row and counts
 // the matching prefix of every sequence.  In the streaming form it needs no launch of its own:
-// the warp that delivers the last chunk of a row (one atomicAdd on a per-row counter that
-// started at zero) folds that row, and the warp that folds the last row of all counts the
-// prefixes -- nobody waits for anybody.  Ordering rule everywhere: a NaN beats any
+// when a CTA has delivered all its candidates, its threads count them on per-row counters that
+// started at zero; the thread whose count completes a row folds that row, and the CTA in which
+// the last row of all was completed counts the prefixes -- nobody waits for anybody.  Ordering
+// rule everywhere: a NaN beats any
 // number, larger value beats smaller, equal values (and two NaNs) go to the lower
 // index -- the lowest-index-of-the-maximum convention with NaN treated as maximal.
 #include <limits.h>
@@ -107,7 +108,7 @@ constexpr int kStages = 6;                       // 32 KB chunks in flight per S
 constexpr int kStreamWarps = kStages;             // warp w owns stage w: it follows that stage's barrier phase by phase
 constexpr int kStreamThreads = (kStreamWarps + 1) * 32;
 constexpr int kStageBytes = kChunk * 4;
-constexpr int kStreamSmem = kStages * kStageBytes + 2 * kStages * 8 + 16;
+constexpr int kStreamSmem = kStages * kStageBytes + 2 * kStages * 8 + 32;
 
 // Set (to a magic word) if a wait inside the streaming kernel ever ran into its time limit; the
 // candidates of the chunks that were not finished then carry index -1, which matches no draft.
@@ -144,44 +145,51 @@ __device__ __forceinline__ int match_prefix(const int32_t* __restrict__ draft, c
   return m;
 }
 
-// Called by a whole warp after it has delivered `part[row * n_chunks + chunk]`.
-__device__ __forceinline__ void accept_tail(const Tail& t, const Cand* part, int n_chunks, int row, int lane) {
-  unsigned int prev = 0;
-  if (lane == 0) {
-    __threadfence();                                   // the candidate is visible before the count
-    prev = atomicAdd(t.cnt + row, 1u);
-  }
-  prev = __shfl_sync(0xffffffffu, prev, 0);
-  if (prev + 1u != static_cast<unsigned int>(n_chunks)) return;
-  // every chunk of this row is in: fold them
-  __threadfence();
-  Cand best{-INFINITY, INT_MAX};
-  const Cand* pr = part + static_cast<int64_t>(row) * n_chunks;
-  for (int c = lane; c < n_chunks; c += 32) {
-    const Cand x = load_cand(pr + c);
-    if (x.i < 0) { best.v = NAN; best.i = -1; }        // an unfinished chunk: the row matches no draft
-    else if (best.i != -1) fold(best, x.v, x.i);
-  }
-  const bool bad = __any_sync(0xffffffffu, best.i == -1);
-  best = warp_best(best);
-  unsigned int rows_done = 0;
-  if (lane == 0) {
+// Pass 2 inside pass 1, run by the kStreamWarps consumer warps of a CTA once all of them have
+// delivered their candidates: every thread counts one of the CTA's items on the item's row; the
+// thread whose count completes a row folds that row's candidates and counts the row; the CTA in
+// which the last row of all was completed counts every sequence's matching prefix.  One round of
+// atomics per CTA, no per-item stall, and nobody waits for another CTA.
+__device__ __forceinline__ void accept_tail(const Tail& t, const Cand* part, int n_chunks, int n_local, int n_items,
+                                            volatile int* s_last) {
+  const int tid = threadIdx.x, n_thr = kStreamWarps * 32;
+  __threadfence();                                       // this thread's candidates are visible device-wide
+  asm volatile("bar.sync 1, %0;" ::"r"(n_thr) : "memory");
+  for (int k = tid; k < n_local; k += n_thr) {
+    const int item = static_cast<int>(blockIdx.x) + k * static_cast<int>(gridDim.x);
+    const int row = item / n_chunks;
+    if (atomicAdd(t.cnt + row, 1u) + 1u != static_cast<unsigned int>(n_chunks)) continue;
+    // every chunk of this row is in: fold them
+    __threadfence();
+    Cand best{-INFINITY, INT_MAX};
+    bool bad = false;
+    const Cand* pr = part + static_cast<int64_t>(row) * n_chunks;
+    for (int c0 = 0; c0 < n_chunks; c0 += 8) {          // eight loads in flight, then the folds
+      Cand p[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) p[u] = (c0 + u < n_chunks) ? load_cand(pr + c0 + u) : Cand{-INFINITY, INT_MAX};
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        bad |= (p[u].i < 0);                             // an unfinished chunk: the row matches no draft
+        fold(best, p[u].v, p[u].i);
+      }
+    }
     t.argmax_out[row] = bad ? -1 : best.i;
     t.cnt[row] = 0u;
     __threadfence();
-    rows_done = atomicAdd(t.cnt + t.T, 1u);
+    if (atomicAdd(t.cnt + t.T, 1u) + 1u == static_cast<unsigned int>(t.T)) *s_last = 1;
   }
-  rows_done = __shfl_sync(0xffffffffu, rows_done, 0);
-  if (rows_done + 1u != static_cast<unsigned int>(t.T)) return;
+  asm volatile("bar.sync 1, %0;" ::"r"(n_thr) : "memory");
+  if (!*s_last) return;
   // every row has its argmax: the prefix of every sequence
   __threadfence();
-  for (int b = lane; b < t.B; b += 32) {
+  for (int b = tid; b < t.B; b += n_thr) {
     const int r0 = t.row_off[b], r1 = t.row_off[b + 1];
     const int m = match_prefix(t.draft, t.argmax_out, r0, r1);
     t.n_match[b] = m;
     if (t.n_keep) t.n_keep[b] = (r1 > r0) ? m + 1 : 0;
   }
-  if (lane == 0) t.cnt[t.T] = 0u;
+  if (tid == 0) t.cnt[t.T] = 0u;
 }
 
 __global__ void __launch_bounds__(kStreamThreads, 1)
@@ -198,6 +206,7 @@ argmax_stream_kernel(const float* __restrict__ logits, int64_t ld_v, int V, int 
       ms::mbar_init(bars + 8 * (kStages + i), 1);
     }
     ms::wait_ctx_init(abort_flag, wait_limit_us);
+    abort_flag[4] = 0;                                   // "this CTA completed the last row"
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
@@ -301,8 +310,8 @@ argmax_stream_kernel(const float* __restrict__ logits, int64_t ld_v, int V, int 
       best.i = -1;
     }
     if (lane == 0) part[item] = best;
-    if (tail.cnt) accept_tail(tail, part, n_chunks, row, lane);
   }
+  if (tail.cnt) accept_tail(tail, part, n_chunks, n_local, n_items, abort_flag + 4);
 }
 
 __global__ void __launch_bounds__(128)
