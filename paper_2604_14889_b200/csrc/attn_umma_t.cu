@@ -586,7 +586,10 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
         float l_row[CW];
 #pragma unroll
         for (int j = 0; j < CW; ++j) l_row[j] = (red_g[j] + red_g[32 + j]) + (red_g[64 + j] + red_g[96 + j]);
+        // thread t < CW also owns the statistics of row c0 + t (written once, outside the row loop below,
+        // where a per-row "if (t == j)" made one warp walk 32 divergent branches)
         const float m_mine = (t < CW) ? mref_g[t] : 0.f;
+        const float l_mine = (t < CW) ? (red_g[t] + red_g[32 + t]) + (red_g[64 + t] + red_g[96 + t]) : 1.f;
         if (!wg_sync()) { ok = false; break; }          // red and m_ref may be reused from here on
         if (!wait_all(bars + 8 * (kTbPvDone + pb), (it >> 1) & 1)) { ok = false; break; }
         tc_fence_after();
@@ -607,9 +610,13 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
           for (int j = 0; j < CW; ++j) {
             if (c0 + j < rows) {
               out_l[orow * D + t] = __float2bfloat16_rn(__uint_as_float(o[j]) * __frcp_rn(l_row[j]));
-              if (lse_l && t == j) lse_l[orow] = (m_mine + log2f(l_row[j])) * 0.69314718055994531f;
             }
             if (++g == a.G) { g = 0; orow += next_token; } else { ++orow; }
+          }
+          if (lse_l && t < CW && c0 + t < rows) {
+            const int r = c0 + t, i = r / a.G;
+            lse_l[static_cast<int64_t>(w.r0 + i) * a.H_q + w.h * a.G + (r - i * a.G)] =
+                (m_mine + log2f(l_mine)) * 0.69314718055994531f;
           }
         } else {
           float* slot = ws_slots + static_cast<size_t>(w.slot) * ws_slot_floats(D, rows_pad);
@@ -618,11 +625,11 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
           for (int j = 0; j < CW; ++j) {
             if (c0 + j < rows) {
               slot[static_cast<size_t>(c0 + j) * D + t] = __uint_as_float(o[j]);
-              if (t == j) {
-                sm[c0 + j] = m_mine;
-                sm[rows_pad + c0 + j] = l_row[j];
-              }
             }
+          }
+          if (t < CW && c0 + t < rows) {
+            sm[c0 + t] = m_mine;
+            sm[rows_pad + c0 + t] = l_mine;
           }
           if (a.done) {
             // The unit is cut across CTAs.  Each warpgroup of each of its CTAs counts itself once its
