@@ -260,6 +260,15 @@ MS_API int32_t memosight_attn_status(const void* workspace, memosight_stream_t s
  * memosight_attn_status(workspace) then reports MS_ERR_DEVICE_TIMEOUT once -- the whole failure
  * path exercised without anything failing.  workspace: device, 256-byte aligned, >= 256 bytes. */
 MS_API uint32_t memosight_debug_set_wait_limit_us(uint32_t limit_us);
+/* Several calls finish their work in the tail of their main kernel (the merge of cut attention
+ * units, pass 2 of the accept, the new lengths of append / compaction / keep-list eviction): the
+ * block that finishes last does it, which it learns from a counter in a fixed array inside the
+ * library (128 banks of counters, handed out per buffer address; 1 MB on every GPU that loads the
+ * library).  A call that gets no bank uses its two-launch form instead, with the same result.
+ * memosight_debug_set_bank_limit caps the number of banks handed out from now on (0: every call
+ * takes the two-launch form; buffers that already own a bank below the cap keep it) and returns
+ * the previous cap; a negative value only queries.  For tests of the two-launch forms. */
+MS_API int32_t memosight_debug_set_bank_limit(int32_t n_banks);
 MS_API int32_t memosight_debug_wait_timeout(void* workspace, uint32_t limit_us, memosight_stream_t stream);
 
 /* ---- KV compaction and append (Sec. 2.1.2; Algorithm 1: UpdateCache, S <- S (+) A) ------- */

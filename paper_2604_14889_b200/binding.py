@@ -144,6 +144,8 @@ def lib() -> C.CDLL:
         L.memosight_attn_debug_events.argtypes = [C.c_void_p, C.c_void_p]
         L.memosight_debug_set_wait_limit_us.restype = C.c_uint32
         L.memosight_debug_set_wait_limit_us.argtypes = [C.c_uint32]
+        L.memosight_debug_set_bank_limit.restype = C.c_int32
+        L.memosight_debug_set_bank_limit.argtypes = [C.c_int32]
         L.memosight_debug_wait_timeout.restype = C.c_int32
         L.memosight_debug_wait_timeout.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p]
         L.memosight_attn_set_path.restype = C.c_int32
@@ -335,6 +337,12 @@ def memosight_attn_set_path(path: int) -> int:
 def memosight_debug_set_wait_limit_us(limit_us: int) -> int:
     """Limit of one bounded device-side wait for later launches; returns the previous one (0 only queries)."""
     return int(lib().memosight_debug_set_wait_limit_us(int(limit_us)))
+
+
+def memosight_debug_set_bank_limit(n_banks: int) -> int:
+    """Caps the last-block-done counter banks handed out (0: every call takes its two-launch form);
+    returns the previous cap; negative only queries."""
+    return int(lib().memosight_debug_set_bank_limit(int(n_banks)))
 
 
 def memosight_debug_wait_timeout(workspace, limit_us: int, stream=None) -> None:

@@ -34,6 +34,7 @@ struct DeviceBanks {
 
 std::mutex g_mu;
 DeviceBanks g_banks[kMaxDevices];
+int g_bank_limit = kDoneBanks;      // memosight_debug_set_bank_limit
 
 }  // namespace
 
@@ -51,9 +52,10 @@ unsigned int* done_bank(const void* key) {
     }
     d.base = static_cast<unsigned int*>(p);
   }
-  for (int i = d.used - 1; i >= 0; --i)
+  const int limit = g_bank_limit < kDoneBanks ? g_bank_limit : kDoneBanks;
+  for (int i = (d.used < limit ? d.used : limit) - 1; i >= 0; --i)
     if (d.key[i] == key) return d.base + static_cast<size_t>(i) * kDoneBankWords;
-  if (d.used == kDoneBanks) return nullptr;
+  if (d.used >= limit) return nullptr;
   d.key[d.used] = key;
   return d.base + static_cast<size_t>(d.used++) * kDoneBankWords;
 }
@@ -66,3 +68,10 @@ int32_t done_bank_clear(const void* key, cudaStream_t st) {
 }
 
 }  // namespace ms
+
+extern "C" int32_t memosight_debug_set_bank_limit(int32_t n_banks) {
+  std::lock_guard<std::mutex> lock(ms::g_mu);
+  const int32_t prev = ms::g_bank_limit;
+  if (n_banks >= 0) ms::g_bank_limit = n_banks;
+  return prev;
+}

@@ -108,3 +108,26 @@ def test_step_host_equals_the_separate_calls_two_steps():
     assert torch.equal(h_am, want[1]["am"].cpu()) and torch.equal(h_nm, want[1]["nm"].cpu())
     assert torch.equal(inp.kv_len, want[1]["len"])
     assert torch.equal(inp.k_cache, want[1]["k"]) and torch.equal(inp.v_cache, want[1]["v"])
+
+    # ---- and once more with no host buffers at all: the whole device-resident step queued by one call.
+    #      The step's tensors are put into the device staging buffers beforehand; nothing is copied.
+    inp.k_cache.copy_(snap["k"])
+    inp.v_cache.copy_(snap["v"])
+    inp.kv_len.copy_(snap["len"])
+    g["out"].zero_()
+    for name in ("h_q", "h_k_step", "h_v_step", "h_pos_id", "h_logits", "h_draft", "h_out", "h_argmax", "h_n_match"):
+        setattr(p, name, None)
+    d_pos.copy_(pos)
+    for s in range(2):
+        d_q.copy_(inp.q)
+        d_ks.copy_(inp.k_step)
+        d_vs.copy_(inp.v_step)
+        p.d_logits, p.d_draft = accs[s].logits.data_ptr(), accs[s].draft.data_ptr()
+        p.d_seg_start, p.d_seg_len = (seg_start.data_ptr(), seg_len.data_ptr()) if s == 0 else (None, None)
+        ms.memosight_step_host(p)
+    torch.cuda.synchronize()
+    assert ms.memosight_attn_status(g["ws"]) == ms.MS_OK
+    assert torch.equal(g["out"], want[1]["out"])
+    assert torch.equal(g["am"], want[1]["am"]) and torch.equal(g["nm"], want[1]["nm"])
+    assert torch.equal(inp.kv_len, want[1]["len"])
+    assert torch.equal(inp.k_cache, want[1]["k"]) and torch.equal(inp.v_cache, want[1]["v"])
