@@ -30,17 +30,19 @@ constexpr int kBCw = kTile / kBWg;
 constexpr int kBThreads = 128 + 128 * kBWg;       // warp 0: TMA, warp 1: MMA issue, warps 4..: softmax warpgroups
 constexpr int kBD = 128;
 static_assert(kBCw % 32 == 0 && kBD / kBWg == kBCw, "a warpgroup's score and output columns are whole 32-column loads");
-constexpr uint32_t kBCols = 512;  // S0 | S1 | O
-constexpr uint32_t kBColS = 0, kBColO = 256;
+constexpr uint32_t kBCols = 512;  // S0 | S1 | O of key columns 0..63 | O of key columns 64..127
+constexpr uint32_t kBColS = 0, kBColO = 256;      // accumulator of softmax warpgroup g at kBColO + g * kBD
+static_assert(kBWg == 2 && kBColO + kBWg * kBD <= kBCols, "one output accumulator per softmax warpgroup");
 constexpr float kBGrowSum = 281474976710656.f;   // 2^48: a partial row sum this large moves the reference
 constexpr int kBKv = 4;                           // K/V buffers in the ring
 constexpr int kBKvBytes = kTile * kBD * 2;        // 32 KB
 constexpr uint32_t kBHalf = kTile * 128;          // bytes between 64-column halves of a tile
-constexpr int kBQBytes = 2 * kBHalf, kBPBytes = 2 * kBHalf;
-constexpr int kBOffQ = 0, kBOffP = kBQBytes, kBOffKv = kBOffP + 2 * kBPBytes;
+constexpr int kBQBytes = 2 * kBHalf;
+constexpr int kBOffQ = 0, kBOffKv = kBQBytes;
 constexpr int kBOffMisc = kBOffKv + kBKv * kBKvBytes;
-// misc: barriers | scalars | mx[kBWg][128] and lpart[kBWg][128] (one region: they are never live together)
-constexpr int kBMiscScalars = 256, kBMiscMx = 512, kBMiscL = 512, kBMiscBytes = 512 + kBWg * kTile * 4;
+// misc: barriers | scalars | mx[kBWg][128] | lpart[kBWg][128]
+constexpr int kBMiscScalars = 256, kBMiscMx = 512, kBMiscL = kBMiscMx + kBWg * kTile * 4;
+constexpr int kBMiscBytes = kBMiscL + kBWg * kTile * 4;
 constexpr int kBSmem = kBOffMisc + kBMiscBytes;
 static_assert(kBSmem <= 227 * 1024, "shared memory budget");
 
@@ -247,9 +249,8 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
   const uint32_t bars = sb + kBOffMisc;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kBOffMisc + kBMiscScalars);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kBOffMisc + kBMiscScalars + 8);
-  volatile int* grow_flag = reinterpret_cast<volatile int*>(smem + kBOffMisc + kBMiscScalars + 16);
   float* s_mx = reinterpret_cast<float*>(smem + kBOffMisc + kBMiscMx);      // [kBWg][128]
-  float* s_lp = reinterpret_cast<float*>(smem + kBOffMisc + kBMiscL);       // [kBWg][128], same memory
+  float* s_lp = reinterpret_cast<float*>(smem + kBOffMisc + kBMiscL);       // [kBWg][128]
   uint32_t* status = reinterpret_cast<uint32_t*>(a.workspace);
   int* ws_pre = reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(a.workspace) + kWsHeaderBytes);
   float* ws_slots = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(a.workspace) + kWsHeaderBytes +
@@ -286,7 +287,6 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
     mbar_init(bars + 8 * kBbAll, 4 * kBWg);
     mbar_init(bars + 8 * kBbDrain, 1);
     wait_ctx_init(abort_flag, a.wait_limit_us);
-    *grow_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
@@ -394,12 +394,23 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
     // =========================== MMA issuer ===========================
     const uint32_t idesc_qk = instr_desc(kTile, 0), idesc_pv = instr_desc(D, 1);
     const uint32_t q_lo = desc_lo(sb + kBOffQ, 16), k_lo0 = desc_lo(sb + kBOffKv, 16);
-    const uint32_t p_lo0 = desc_lo(sb + kBOffP, 16), v_lo0 = desc_lo(sb + kBOffKv, kBHalf);
+    const uint32_t v_lo0 = desc_lo(sb + kBOffKv, kBHalf);
     BigWalk wq = w0, wp = w0;
     RingPos rk, rv;
     rk.init(0, kBKv);
     rv.init(1, kBKv);
     bool ok = true;
+    // Keys 0..63 of a tile accumulate into the first output accumulator, keys 64..127 into the
+    // second: each softmax warpgroup then owns the running reference of its own accumulator and
+    // the two never have to agree inside an item.  The second accumulator is first written by the
+    // item's first tile with more than 64 valid keys.
+    bool o1_live = false;
+    // P of 16 keys = 8 columns of tensor memory: warpgroup g left its 64 keys in the first 32 of its
+    // 64 score columns
+    auto issue_pv = [&](const uint32_t p_col, const uint32_t v_lo, const int j, const uint32_t acc) {
+      umma_bf16_ts_lo(tmem + kBColO + (j >> 2) * kBD, p_col + (j >> 2) * kBCw + (j & 3) * 8,
+                      v_lo + j * (2048 >> 4), idesc_pv, acc);
+    };
     auto issue_qk = [&]() -> bool {
       bwalk_tile(wq);
       const int it = wq.it;
@@ -452,12 +463,12 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
           }
           tc_fence_after();
           {
-            const uint32_t p_lo = p_lo0 + (it & 1) * (kBPBytes >> 4);
+            const uint32_t p_lo = tmem + kBColS + (it & 1) * kTile;
             const uint32_t v_lo = v_lo0 + rv.buf * (kBKvBytes >> 4);
+            const uint32_t acc1 = o1_live ? 1u : 0u;
 #pragma unroll
-            for (int j = 0; j < kTile / 16; ++j)
-              umma_bf16_lo(tmem + kBColO, p_lo + (j >> 2) * (kBHalf >> 4) + (j & 3) * 2, v_lo + j * (2048 >> 4),
-                           idesc_pv, 1u);
+            for (int j = 0; j < kTile / 16; ++j) issue_pv(p_lo, v_lo, j, j == 4 ? acc1 : 1u);
+            o1_live = true;
             umma_commit(bars + 8 * (kBbKvEmpty + rv.buf));
             rv.step(2);
           }
@@ -480,21 +491,20 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
         break;
       }
       tc_fence_after();
-      const uint32_t p_lo = p_lo0 + (it & 1) * (kBPBytes >> 4);
+      const uint32_t p_lo = tmem + kBColS + (it & 1) * kTile;
       const uint32_t v_lo = v_lo0 + rv.buf * (kBKvBytes >> 4);
       const int ksteps = (wp.nvalid + 15) >> 4;
       const uint32_t acc0 = wp.first ? 0u : 1u;
+      if (wp.first) o1_live = false;
+      const uint32_t acc1 = o1_live ? 1u : 0u;
       if (ksteps == kTile / 16) {
 #pragma unroll
-        for (int j = 0; j < kTile / 16; ++j)
-          umma_bf16_lo(tmem + kBColO, p_lo + (j >> 2) * (kBHalf >> 4) + (j & 3) * 2, v_lo + j * (2048 >> 4),
-                       idesc_pv, j == 0 ? acc0 : 1u);
+        for (int j = 0; j < kTile / 16; ++j) issue_pv(p_lo, v_lo, j, j == 0 ? acc0 : (j == 4 ? acc1 : 1u));
       } else {
 #pragma unroll 1
-        for (int j = 0; j < ksteps; ++j)
-          umma_bf16_lo(tmem + kBColO, p_lo + (j >> 2) * (kBHalf >> 4) + (j & 3) * 2, v_lo + j * (2048 >> 4),
-                       idesc_pv, j == 0 ? acc0 : 1u);
+        for (int j = 0; j < ksteps; ++j) issue_pv(p_lo, v_lo, j, j == 0 ? acc0 : (j == 4 ? acc1 : 1u));
       }
+      if (ksteps > 4) o1_live = true;
       umma_commit(bars + 8 * (kBbKvEmpty + rv.buf));
       rv.step(2);
       bwalk_next(a, wp, pre);
@@ -506,14 +516,17 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
       }
     }
   } else if (warp >= 4 && n_iter > 0) {
-    // ====== softmax warps: thread = packed row; warpgroup g = key columns / output columns [kBCw*g, kBCw*(g+1)) ======
+    // ====== softmax warps: thread = packed row; warpgroup g = key columns [kBCw*g, kBCw*(g+1)) of every tile, with
+    //        an output accumulator and a running reference of its own.  Inside an item the two groups
+    //        never talk; at its end they fold their halves and group g writes output columns
+    //        [kBCw*g, kBCw*(g+1)) ======
     const int wg = (warp - 4) >> 2, quad = (warp - 4) & 3;
     const int r = quad * 32 + lane;
     const uint32_t lane_addr = tmem + (static_cast<uint32_t>(quad * 32) << 16);
-    const uint32_t rx = r & 7;
     BigWalk w = w0;
     float m_ref = 0.f, l_part = 0.f;
-    bool unref = false;     // the row has not seen a visible key in this item yet: it has no reference
+    bool unref = false;     // the row has not seen a visible key among this group's columns in this item: no reference yet
+    bool o1_live = false;   // the second accumulator has been written in this item (a tile with more than 64 valid keys)
     int tok = 0, anc = 0, rows = 0;
     bool row_ok = false;
     uint32_t all_phase = 0;
@@ -536,12 +549,6 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
       const bool good = wait_all(bars + 8 * kBbAll, all_phase & 1);
       ++all_phase;
       return good;
-    };
-    auto max_of_groups = [&](const float* arr) -> float {
-      float m = arr[r];
-#pragma unroll
-      for (int g = 1; g < kBWg; ++g) m = fmaxf(m, arr[g * kTile + r]);
-      return m;
     };
     // One tile from the scores in tensor memory to P handed over (S(it) is complete; the P buffer is
     // free with it: the commit behind S(it) tracks every earlier tcgen05 operation of the issuing
@@ -577,42 +584,37 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
       } else
         big_load_scores<false>(s_addr, v, 0, kTile, false, 0, 0, 0, 0);
       if (opens_item) {
-        // new unit: reference = exact maximum of the first tile over all column groups
-        s_mx[wg * kTile + r] = max_cols(v);
-        if (!sync_all()) return false;
-        const float m = max_of_groups(s_mx);
-        // A row that sees no key in the item's first tile (a chunk that starts right of the row's
-        // causal limit, a foresight row with anchor 0, a training-mask row behind other steps' tokens)
-        // stays without a reference: the first later tile with a visible key sets it through the
-        // branch below, whatever the size of its scores (a placeholder of 0 would flush strongly
-        // negative rows to a zero sum).
+        // new item: reference = exact maximum of the first tile over this group's columns
+        const float m = max_cols(v);
+        // A row that sees no key there (a chunk that starts right of the row's causal limit, a
+        // foresight row with anchor 0, a training-mask row behind other steps' tokens, the right
+        // half of a diagonal tile) stays without a reference: the first later tile with a visible
+        // key sets it through the branch below, whatever the size of its scores (a placeholder of
+        // 0 would flush strongly negative rows to a zero sum).
         unref = (m == -INFINITY);
         m_ref = unref ? 0.f : m * a.scale_log2;
         l_part = 0.f;
+        o1_live = false;
       }
-      // p = 2^(s*scale - m_ref) as bf16 into this row of the P tile; the row's partial sum over
-      // this group's keys
-      const uint32_t p_row = sb + kBOffP + pb * kBPBytes + ((wg * kBCw) >> 6) * kBHalf + r * 128;
-      const int chunk0 = ((wg * kBCw) & 63) >> 3;             // first 16-byte chunk inside the 64-key half
+      // p = 2^(s*scale - m_ref) as bf16 over the first half of this thread's own score columns (all
+      // 64 scores are in registers by now), two keys per column; the row's partial sum over this
+      // group's keys
       auto p_pass = [&]() -> float {
         // scale-and-shift and the running sums two values per instruction (packed fp32 pairs)
         const f32x2_t scale2 = pack_f32x2(a.scale_log2, a.scale_log2), nm2 = pack_f32x2(-m_ref, -m_ref);
         f32x2_t ls[2] = {pack_f32x2(0.f, 0.f), pack_f32x2(0.f, 0.f)};
   #pragma unroll
-        for (int c = 0; c < kBCw / 8; ++c) {
-          float p[8];
+        for (int c = 0; c < kBCw / 16; ++c) {
+          uint32_t pk[8];
   #pragma unroll
-          for (int e = 0; e < 8; e += 2) {
+          for (int e = 0; e < 16; e += 2) {
             float x0, x1;
-            unpack_f32x2(fma_f32x2(pack_f32x2(v[c * 8 + e], v[c * 8 + e + 1]), scale2, nm2), x0, x1);
-            p[e] = ex2(x0);
-            p[e + 1] = ex2(x1);
-            ls[(e >> 1) & 1] = add_f32x2(ls[(e >> 1) & 1], pack_f32x2(p[e], p[e + 1]));
+            unpack_f32x2(fma_f32x2(pack_f32x2(v[c * 16 + e], v[c * 16 + e + 1]), scale2, nm2), x0, x1);
+            const float p0 = ex2(x0), p1 = ex2(x1);
+            ls[(e >> 1) & 1] = add_f32x2(ls[(e >> 1) & 1], pack_f32x2(p0, p1));
+            pk[e >> 1] = pack2(p0, p1);
           }
-          const uint32_t addr = p_row + (((chunk0 + c) ^ rx) << 4);
-          asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(pack2(p[0], p[1])),
-                       "r"(pack2(p[2], p[3])), "r"(pack2(p[4], p[5])), "r"(pack2(p[6], p[7]))
-                       : "memory");
+          tmem_st8(s_addr + c * 8, pk);
         }
         float s0, s1, s2, s3;
         unpack_f32x2(ls[0], s0, s1);
@@ -620,40 +622,46 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
         return (s0 + s1) + (s2 + s3);
       };
       float tsum = p_pass();
-      // A score that outgrew the row reference by ~2^48 shows in the sum (so do inf and NaN); the
-      // softmax warps agree on it before anyone hands P over
-      bool regrow = row_ok && !(tsum < kBGrowSum);
-      if (unref && row_ok) regrow = max_cols(v) > -INFINITY;       // the row's first visible key: set its reference
-      if (!opens_item && __any_sync(0xffffffffu, regrow) && lane == 0) *grow_flag = it + 1;
-      if (!sync_all()) return false;
-      if (*grow_flag == it + 1) {
-        // ---- rare: move the row references up; rescale O (this group's columns) and the sums ----
-        s_mx[wg * kTile + r] = max_cols(v);
-        if (!sync_all()) return false;
-        const float m = max_of_groups(s_mx);
-        const float m_new = (m == -INFINITY) ? m_ref : (unref ? m * a.scale_log2 : fmaxf(m_ref, m * a.scale_log2));
-        // (a row without a reference has accumulated nothing: its O and sum are zero and stay so)
-        const float alpha = unref ? 1.f : ex2(m_ref - m_new);
-        if (m != -INFINITY) unref = false;
-        m_ref = m_new;
-        l_part *= alpha;
-        if (!wait_all(bar_pv_done(it - 1), ((it - 1) >> 1) & 1)) return false;
-        tc_fence_after();
-  #pragma unroll 1
-        for (int c = 0; c < kBCw / 32; ++c) {
-          uint32_t o[32];
-          tmem_ld32(lane_addr + kBColO + wg * kBCw + c * 32, o);
-          tmem_ld_wait(o);
-  #pragma unroll
-          for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-          tmem_st32(lane_addr + kBColO + wg * kBCw + c * 32, o);
+      // A score that outgrew the row reference by ~2^48 shows in the sum (so do inf and NaN).  The
+      // reference belongs to this thread alone -- its 64 key columns, its accumulator -- so the
+      // decision is the thread's own; only the tensor-memory accesses need the whole warp.
+      bool regrow = row_ok && !opens_item && !(tsum < kBGrowSum);
+      if (unref && row_ok && !opens_item) regrow = max_cols(v) > -INFINITY;   // the row's first visible key here: set its reference
+      if (__any_sync(0xffffffffu, regrow)) {
+        // ---- rare: move row references up; rescale this group's accumulator and sums ----
+        float alpha = 1.f;
+        if (regrow) {
+          const float m = max_cols(v) * a.scale_log2;
+          // (a row without a reference has accumulated nothing: its O and sum are zero and stay so)
+          const float m_new = unref ? m : fmaxf(m_ref, m);
+          alpha = unref ? 1.f : ex2(m_ref - m_new);
+          unref = false;
+          m_ref = m_new;
+          l_part *= alpha;
         }
-        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+        if (wg == 0 || o1_live) {
+          if (!wait_all(bar_pv_done(it - 1), ((it - 1) >> 1) & 1)) return false;
+          tc_fence_after();
+  #pragma unroll 1
+          for (int c = 0; c < kBD / 32; ++c) {
+            uint32_t o[32];
+            tmem_ld32(lane_addr + kBColO + wg * kBD + c * 32, o);
+            tmem_ld_wait(o);
+  #pragma unroll
+            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+            tmem_st32(lane_addr + kBColO + wg * kBD + c * 32, o);
+          }
+          asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+        }
+        // every lane again: the stores to tensor memory are warp-wide instructions (a lane whose
+        // reference stayed writes the same values as before)
+        __syncwarp();
         tsum = p_pass();
-        if (!sync_all()) return false;     // s_mx may be rewritten from here on
       }
+      if (nv > kBCw) o1_live = true;
       l_part += tsum;
-      fence_async_smem();
+      asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+      if (masked && (nv & 15)) fence_async_smem();     // the cleared V rows, for the tensor core
       tc_fence_before();
       __syncwarp();
       mbar_arrive_if(lane == 0, bars + 8 * (kBbPFull + pb));
@@ -704,32 +712,46 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
       }
 
       if (w.last) {
-        // ---- end of the item: the unit, or this chunk of it ----
+        // ---- end of the item: the unit, or this chunk of it.  Fold the two groups' halves:
+        //      (m_g, l_g, O_g) relative to M = max m_g; a group that saw no key counts as m = -inf
+        s_mx[wg * kTile + r] = (unref || !(wg == 0 || o1_live)) ? -INFINITY : m_ref;
         s_lp[wg * kTile + r] = l_part;
         if (!sync_all()) { ok = false; break; }
-        float l_row = 0.f;
-#pragma unroll
-        for (int g = 0; g < kBWg; ++g) l_row += s_lp[g * kTile + r];
+        const float m0 = s_mx[r], m1 = s_mx[kTile + r];
+        const float m_row = fmaxf(m0, m1);
+        const float w0 = (m0 == -INFINITY) ? 0.f : ex2(m0 - m_row);
+        const float w1 = (m1 == -INFINITY) ? 0.f : ex2(m1 - m_row);
+        const float l_row = s_lp[r] * w0 + s_lp[kTile + r] * w1;
         if (!wait_all(bar_pv_done(it), (it >> 1) & 1)) { ok = false; break; }
         tc_fence_after();
         const int i = tok, g = r % a.G;
         const int64_t orow = static_cast<int64_t>(w.s.r0 + (row_ok ? i : 0)) * a.H_q + w.h * a.G + g;
         float* slot = ws_slots + static_cast<size_t>(w.slot < 0 ? 0 : w.slot) * big_slot_floats();
-        const float inv = 1.f / l_row;
+        const float inv = (w.slot < 0) ? 1.f / l_row : 1.f;     // a partial stays unnormalised, relative to m_row
+        const float f0 = w0 * inv, f1 = w1 * inv;
 #pragma unroll 1
         for (int c = 0; c < kBCw / 32; ++c) {
           uint32_t o[32];
           tmem_ld32(lane_addr + kBColO + wg * kBCw + c * 32, o);
           tmem_ld_wait(o);
+#pragma unroll
+          for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * f0);
+          if (o1_live) {
+            uint32_t o1[32];
+            tmem_ld32(lane_addr + kBColO + kBD + wg * kBCw + c * 32, o1);
+            tmem_ld_wait(o1);
+#pragma unroll
+            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(fmaf(__uint_as_float(o1[e]), f1, __uint_as_float(o[e])));
+          }
           if (row_ok && w.slot < 0) {
             uint4* op = reinterpret_cast<uint4*>(a.out + orow * D + wg * kBCw + c * 32);
 #pragma unroll
             for (int q4 = 0; q4 < 4; ++q4) {
               uint4 u;
-              u.x = pack2(__uint_as_float(o[8 * q4 + 0]) * inv, __uint_as_float(o[8 * q4 + 1]) * inv);
-              u.y = pack2(__uint_as_float(o[8 * q4 + 2]) * inv, __uint_as_float(o[8 * q4 + 3]) * inv);
-              u.z = pack2(__uint_as_float(o[8 * q4 + 4]) * inv, __uint_as_float(o[8 * q4 + 5]) * inv);
-              u.w = pack2(__uint_as_float(o[8 * q4 + 6]) * inv, __uint_as_float(o[8 * q4 + 7]) * inv);
+              u.x = pack2(__uint_as_float(o[8 * q4 + 0]), __uint_as_float(o[8 * q4 + 1]));
+              u.y = pack2(__uint_as_float(o[8 * q4 + 2]), __uint_as_float(o[8 * q4 + 3]));
+              u.z = pack2(__uint_as_float(o[8 * q4 + 4]), __uint_as_float(o[8 * q4 + 5]));
+              u.w = pack2(__uint_as_float(o[8 * q4 + 6]), __uint_as_float(o[8 * q4 + 7]));
               op[q4] = u;
             }
           } else if (row_ok) {
@@ -740,15 +762,16 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
         }
         if (row_ok && wg == 0) {
           if (w.slot < 0) {
-            if (a.lse) a.lse[orow] = (m_ref + log2f(l_row)) * 0.69314718055994531f;
+            if (a.lse) a.lse[orow] = (m_row + log2f(l_row)) * 0.69314718055994531f;
           } else {
+            // a row that saw no key in this chunk leaves m = -inf, l = 0 and a zero O: the merge skips it
             float* sm = slot + static_cast<size_t>(kTile) * D;
-            sm[r] = m_ref;
+            sm[r] = m_row;
             sm[kTile + r] = l_row;
           }
         }
         tc_fence_before();   // the reads of O are ordered before the next item's first PV product
-        if (!sync_all()) { ok = false; break; }   // s_lp and s_mx share their memory with the next item
+        if (!sync_all()) { ok = false; break; }   // s_mx and s_lp are rewritten at the end of the next item
       }
       bwalk_next(a, w, pre);
     }
