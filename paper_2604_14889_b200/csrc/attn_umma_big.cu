@@ -34,7 +34,7 @@ constexpr uint32_t kBCols = 512;  // S0 | S1 | O of key columns 0..63 | O of key
 constexpr uint32_t kBColS = 0, kBColO = 256;      // accumulator of softmax warpgroup g at kBColO + g * kBD
 static_assert(kBWg == 2 && kBColO + kBWg * kBD <= kBCols, "one output accumulator per softmax warpgroup");
 constexpr float kBGrowSum = 281474976710656.f;   // 2^48: a partial row sum this large moves the reference
-constexpr int kBKv = 4;                           // K/V buffers in the ring
+constexpr int kBKv = 6;                           // K/V buffers in the ring: three tiles in flight
 constexpr int kBKvBytes = kTile * kBD * 2;        // 32 KB
 constexpr uint32_t kBHalf = kTile * 128;          // bytes between 64-column halves of a tile
 constexpr int kBQBytes = 2 * kBHalf;
@@ -531,17 +531,18 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
     bool row_ok = false;
     uint32_t all_phase = 0;
     bool ok = true;
-    // "S(it) is complete" and "O += P V of tile it is complete" need no barriers of their own: the
-    // commits that release the tile's K buffer (ring use 2 it) and V buffer (use 2 it + 1) are those
-    // events, and with four ring buffers the phase parity is (it >> 1) & 1 for both.  A waiter is
-    // never two phases behind: the buffer's next use belongs to tile it + 2, whose S needs this
-    // tile's P handed over and whose PV needs its own.
-    static_assert(kBKv == 4, "the ring position of a tile's K and V buffers is taken from its parity");
-    auto bar_s_full = [&](int it) -> uint32_t { return bars + 8 * (kBbKvEmpty + 2 * (it & 1)); };
-    auto bar_pv_done = [&](int it) -> uint32_t { return bars + 8 * (kBbKvEmpty + 2 * (it & 1) + 1); };
     auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {
       return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, status));
     };
+    // "S(it) is complete" and "O += P V of tile it is complete" need no barriers of their own: the
+    // commits that release the tile's K buffer (ring use 2 it) and V buffer (use 2 it + 1) are those
+    // events.  A waiter is never two phases behind: the buffer's next use belongs to tile
+    // it + kBKv / 2, whose S needs the P of every tile before it handed over and whose PV needs its own.
+    auto wait_released = [&](int use) -> bool {
+      return wait_all(bars + 8 * (kBbKvEmpty + use % kBKv), (use / kBKv) & 1);
+    };
+    auto wait_s_full = [&](int it) -> bool { return wait_released(2 * it); };
+    auto wait_pv_done = [&](int it) -> bool { return wait_released(2 * it + 1); };
     // bounded barrier of all softmax warps (also publishes their shared-memory writes)
     auto sync_all = [&]() -> bool {
       __syncwarp();
@@ -640,7 +641,7 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
           l_part *= alpha;
         }
         if (wg == 0 || o1_live) {
-          if (!wait_all(bar_pv_done(it - 1), ((it - 1) >> 1) & 1)) return false;
+          if (!wait_pv_done(it - 1)) return false;
           tc_fence_after();
   #pragma unroll 1
           for (int c = 0; c < kBD / 32; ++c) {
@@ -676,7 +677,7 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
         const int stop = min(w.ti_hi - 1, w.ti < ct ? w.s.L / kTile : ct + big_plain_step_tiles(a, w.s, w.rt, tpt));
         while (w.ti < stop) {
           const int it = w.it;
-          if (!wait_all(bar_s_full(it), (it >> 1) & 1) ||
+          if (!wait_s_full(it) ||
               !tile_body(false, false, kTile, false, 0, it)) {
             ok = false;
             break;
@@ -703,7 +704,7 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
           anc = 0;
         }
       }
-      if (!wait_all(bar_s_full(it), (it >> 1) & 1)) { ok = false; break; }
+      if (!wait_s_full(it)) { ok = false; break; }
       {
         const int nv = w.nvalid;
         const bool is_step = w.step_idx >= 0;
@@ -722,7 +723,7 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
         const float w0 = (m0 == -INFINITY) ? 0.f : ex2(m0 - m_row);
         const float w1 = (m1 == -INFINITY) ? 0.f : ex2(m1 - m_row);
         const float l_row = s_lp[r] * w0 + s_lp[kTile + r] * w1;
-        if (!wait_all(bar_pv_done(it), (it >> 1) & 1)) { ok = false; break; }
+        if (!wait_pv_done(it)) { ok = false; break; }
         tc_fence_after();
         const int i = tok, g = r % a.G;
         const int64_t orow = static_cast<int64_t>(w.s.r0 + (row_ok ? i : 0)) * a.H_q + w.h * a.G + g;
