@@ -52,6 +52,40 @@ enum : int {
 };
 static_assert(kBbCount * 8 <= kBMiscScalars, "barriers overflow their slot");
 
+// The tensor-core instructions as the issuing warp uses them: every lane executes the call with the
+// same operands, the lane that elect.sync names (the same one every time for the full mask) issues.
+__device__ __forceinline__ void umma_bf16_lo_elect(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t idesc,
+                                                   uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p, pe;\n\t.reg .b64 da, db;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "mov.b64 da, {%1, %5};\n\t"
+      "mov.b64 db, {%2, %5};\n\t"
+      "elect.sync _|pe, 0xffffffff;\n\t"
+      "@pe tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}"
+      ::"r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHi)
+      : "memory");
+}
+__device__ __forceinline__ void umma_bf16_ts_lo_elect(uint32_t tmem_d, uint32_t tmem_a, uint32_t b_lo, uint32_t idesc,
+                                                      uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p, pe;\n\t.reg .b64 db;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "mov.b64 db, {%2, %5};\n\t"
+      "elect.sync _|pe, 0xffffffff;\n\t"
+      "@pe tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %3, p;\n\t}"
+      ::"r"(tmem_d), "r"(tmem_a), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHi)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit_elect(uint32_t bar) {
+  asm volatile(
+      "{\n\t.reg .pred pe;\n\t"
+      "elect.sync _|pe, 0xffffffff;\n\t"
+      "@pe tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+      ::"r"(bar)
+      : "memory");
+}
+
 // ---------------------------------------------------------------- schedule
 //
 // Work items are (sequence, KV head, chunk of the unit's tiles, row tile), enumerated in that
@@ -390,8 +424,10 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
     for (int u = uses > kBKv ? uses - kBKv : 0; u < uses; ++u)
       (void)mbar_wait(bars + 8 * (kBbKvFull + u % kBKv), (u / kBKv) & 1, abort_flag, status);
     if (pieces > 0) (void)mbar_wait(bars + 8 * kBbQFull, (pieces - 1) & 1, abort_flag, status);
-  } else if (warp == 1 && lane == 0 && n_iter > 0) {
+  } else if (warp == 1 && n_iter > 0) {
     // =========================== MMA issuer ===========================
+    // The whole warp walks the schedule in step, so that addresses and descriptors are the same in
+    // every lane; one elected lane (always the same one) issues the tensor-core instructions.
     const uint32_t idesc_qk = instr_desc(kTile, 0), idesc_pv = instr_desc(D, 1);
     const uint32_t q_lo = desc_lo(sb + kBOffQ, 16), k_lo0 = desc_lo(sb + kBOffKv, 16);
     const uint32_t v_lo0 = desc_lo(sb + kBOffKv, kBHalf);
@@ -400,6 +436,9 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
     rk.init(0, kBKv);
     rv.init(1, kBKv);
     bool ok = true;
+    auto mwait = [&](uint32_t bar, uint32_t parity) -> bool {
+      return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, status));
+    };
     // Keys 0..63 of a tile accumulate into the first output accumulator, keys 64..127 into the
     // second: each softmax warpgroup then owns the running reference of its own accumulator and
     // the two never have to agree inside an item.  The second accumulator is first written by the
@@ -408,14 +447,14 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
     // P of 16 keys = 8 columns of tensor memory: warpgroup g left its 64 keys in the first 32 of its
     // 64 score columns
     auto issue_pv = [&](const uint32_t p_col, const uint32_t v_lo, const int j, const uint32_t acc) {
-      umma_bf16_ts_lo(tmem + kBColO + (j >> 2) * kBD, p_col + (j >> 2) * kBCw + (j & 3) * 8,
+      umma_bf16_ts_lo_elect(tmem + kBColO + (j >> 2) * kBD, p_col + (j >> 2) * kBCw + (j & 3) * 8,
                       v_lo + j * (2048 >> 4), idesc_pv, acc);
     };
     auto issue_qk = [&]() -> bool {
       bwalk_tile(wq);
       const int it = wq.it;
-      if ((wq.first && !mbar_wait(bars + 8 * kBbQFull, wq.piece_idx & 1, abort_flag, status)) ||
-          !mbar_wait(bars + 8 * (kBbKvFull + rk.buf), rk.par, abort_flag, status))
+      if ((wq.first && !mwait(bars + 8 * kBbQFull, wq.piece_idx & 1)) ||
+          !mwait(bars + 8 * (kBbKvFull + rk.buf), rk.par))
         return false;
       tc_fence_after();
       const uint32_t k_lo = k_lo0 + rk.buf * (kBKvBytes >> 4);
@@ -423,10 +462,10 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
 #pragma unroll
       for (int ks = 0; ks < KSTEPS; ++ks) {
         const uint32_t off = (ks >> 2) * (kBHalf >> 4) + (ks & 3) * 2;
-        umma_bf16_lo(d_s, q_lo + off, k_lo + off, idesc_qk, ks > 0);
+        umma_bf16_lo_elect(d_s, q_lo + off, k_lo + off, idesc_qk, ks > 0);
       }
-      umma_commit(bars + 8 * (kBbKvEmpty + rk.buf));
-      if (wq.last) umma_commit(bars + 8 * kBbQEmpty);
+      umma_commit_elect(bars + 8 * (kBbKvEmpty + rk.buf));
+      if (wq.last) umma_commit_elect(bars + 8 * kBbQEmpty);
       rk.step(2);
       bwalk_next(a, wq, pre);
       return true;
@@ -442,7 +481,7 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
         int it = wp.it;
         for (; n_run > 0; --n_run, ++it) {
           // S(it + 1)
-          if (!mbar_wait(bars + 8 * (kBbKvFull + rk.buf), rk.par, abort_flag, status)) { ok = false; break; }
+          if (!mwait(bars + 8 * (kBbKvFull + rk.buf), rk.par)) { ok = false; break; }
           tc_fence_after();
           {
             const uint32_t k_lo = k_lo0 + rk.buf * (kBKvBytes >> 4);
@@ -450,14 +489,14 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
 #pragma unroll
             for (int ks = 0; ks < KSTEPS; ++ks) {
               const uint32_t off = (ks >> 2) * (kBHalf >> 4) + (ks & 3) * 2;
-              umma_bf16_lo(d_s, q_lo + off, k_lo + off, idesc_qk, ks > 0);
+              umma_bf16_lo_elect(d_s, q_lo + off, k_lo + off, idesc_qk, ks > 0);
             }
-            umma_commit(bars + 8 * (kBbKvEmpty + rk.buf));
+            umma_commit_elect(bars + 8 * (kBbKvEmpty + rk.buf));
             rk.step(2);
           }
           // O += P V (it)
-          if (!mbar_wait(bars + 8 * (kBbPFull + (it & 1)), (it >> 1) & 1, abort_flag, status) ||
-              !mbar_wait(bars + 8 * (kBbKvFull + rv.buf), rv.par, abort_flag, status)) {
+          if (!mwait(bars + 8 * (kBbPFull + (it & 1)), (it >> 1) & 1) ||
+              !mwait(bars + 8 * (kBbKvFull + rv.buf), rv.par)) {
             ok = false;
             break;
           }
@@ -469,7 +508,7 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
 #pragma unroll
             for (int j = 0; j < kTile / 16; ++j) issue_pv(p_lo, v_lo, j, j == 4 ? acc1 : 1u);
             o1_live = true;
-            umma_commit(bars + 8 * (kBbKvEmpty + rv.buf));
+            umma_commit_elect(bars + 8 * (kBbKvEmpty + rv.buf));
             rv.step(2);
           }
         }
@@ -485,8 +524,8 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
       if (wq.it < n_iter && !issue_qk()) { ok = false; break; }
       bwalk_tile(wp);
       const int it = wp.it;
-      if (!mbar_wait(bars + 8 * (kBbPFull + (it & 1)), (it >> 1) & 1, abort_flag, status) ||
-          !mbar_wait(bars + 8 * (kBbKvFull + rv.buf), rv.par, abort_flag, status)) {
+      if (!mwait(bars + 8 * (kBbPFull + (it & 1)), (it >> 1) & 1) ||
+          !mwait(bars + 8 * (kBbKvFull + rv.buf), rv.par)) {
         ok = false;
         break;
       }
@@ -505,12 +544,12 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
         for (int j = 0; j < ksteps; ++j) issue_pv(p_lo, v_lo, j, j == 0 ? acc0 : (j == 4 ? acc1 : 1u));
       }
       if (ksteps > 4) o1_live = true;
-      umma_commit(bars + 8 * (kBbKvEmpty + rv.buf));
+      umma_commit_elect(bars + 8 * (kBbKvEmpty + rv.buf));
       rv.step(2);
       bwalk_next(a, wp, pre);
     }
     if (!ok) {
-      umma_commit(bars + 8 * kBbDrain);
+      umma_commit_elect(bars + 8 * kBbDrain);
       const unsigned long long t_begin = global_ns();
       while (!mbar_try_wait(bars + 8 * kBbDrain, 0) && global_ns() - t_begin < wait_limit_ns(abort_flag)) {
       }
