@@ -9,14 +9,20 @@
 // unit is (sequence, KV head, row tile) and streams the whole cache plus the step-local key
 // tiles up to its own last token (later keys are invisible to all of its rows).
 //
-// Rows on the TMEM lanes: S = Q K^T (128 x 128 per tile) and O += P V on tcgen05.mma, operands
-// from 128-byte-swizzled shared memory filled by TMA, P written by the softmax threads as the
-// K-major A operand.  The softmax is the limit in this compute-heavy regime, so two warpgroups
-// share every tile: warpgroup g takes key columns [64g, 64g+64) of the scores and, for rescales
-// and the epilogue, output columns [64g, 64g+64) of its rows.  A row's reference maximum is the
-// exact maximum of the unit's first tile (both halves, exchanged through shared memory) and only
-// moves when a score exceeds it by about 2^48 (seen in the tile's row sum); the eight softmax warps agree on that through one
-// bounded mbarrier round per tile.  Row sums are kept per thread and added up at the unit's end.
+// Rows on the TMEM lanes: S = Q K^T (128 x 128 per tile, Q and K from 128-byte-swizzled shared
+// memory filled by TMA) and O += P V (P read from tensor memory, V from shared memory) on
+// tcgen05.mma.  The softmax is the limit in this compute-heavy regime, so two warpgroups share
+// every tile: warpgroup g takes key columns [64g, 64g+64) of the scores, writes its P (bf16, two
+// keys per column) over the first half of those same columns once it holds the scores in
+// registers, and owns an output accumulator of its own -- keys 0..63 of every tile accumulate
+// into O_0, keys 64..127 into O_1 -- with its own row references and row sums.  The two groups
+// therefore never have to agree inside an item; at its end they fold (m_g, l_g, O_g) through
+// shared memory and group g writes output columns [64g, 64g+64).  A row's reference is the exact
+// maximum of its group's columns in the item's first tile and only moves when a score exceeds it
+// by about 2^48 (seen in the tile's row sum).  Tensor memory: S0 | S1 | O_0 | O_1 = 512 columns.
+// The whole issuing warp walks the schedule, so that addresses and descriptors are uniform
+// across it, and one elected lane issues: 8 products then issue in ~400 cycles (~620 when a
+// single thread computed them).
 // Schedule: work items dealt round-robin to the persistent CTAs so that the row tiles of one K/V
 // chunk run side by side (see below); every wait is bounded (status word in the workspace, as in
 // the other paths).
@@ -51,40 +57,6 @@ enum : int {
   kBbCount
 };
 static_assert(kBbCount * 8 <= kBMiscScalars, "barriers overflow their slot");
-
-// The tensor-core instructions as the issuing warp uses them: every lane executes the call with the
-// same operands, the lane that elect.sync names (the same one every time for the full mask) issues.
-__device__ __forceinline__ void umma_bf16_lo_elect(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t idesc,
-                                                   uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p, pe;\n\t.reg .b64 da, db;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "mov.b64 da, {%1, %5};\n\t"
-      "mov.b64 db, {%2, %5};\n\t"
-      "elect.sync _|pe, 0xffffffff;\n\t"
-      "@pe tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}"
-      ::"r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHi)
-      : "memory");
-}
-__device__ __forceinline__ void umma_bf16_ts_lo_elect(uint32_t tmem_d, uint32_t tmem_a, uint32_t b_lo, uint32_t idesc,
-                                                      uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p, pe;\n\t.reg .b64 db;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "mov.b64 db, {%2, %5};\n\t"
-      "elect.sync _|pe, 0xffffffff;\n\t"
-      "@pe tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %3, p;\n\t}"
-      ::"r"(tmem_d), "r"(tmem_a), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHi)
-      : "memory");
-}
-__device__ __forceinline__ void umma_commit_elect(uint32_t bar) {
-  asm volatile(
-      "{\n\t.reg .pred pe;\n\t"
-      "elect.sync _|pe, 0xffffffff;\n\t"
-      "@pe tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
-      ::"r"(bar)
-      : "memory");
-}
 
 // ---------------------------------------------------------------- schedule
 //

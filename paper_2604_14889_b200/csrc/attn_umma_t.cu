@@ -230,8 +230,13 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
       (void)mbar_wait(bars + 8 * (kTbKvFull + u % lay.n_kv), (u / lay.n_kv) & 1, abort_flag, status);
     for (int p = pieces > 2 ? pieces - 2 : 0; p < pieces; ++p)
       (void)mbar_wait(bars + 8 * (kTbQFull + (p & 1)), (p >> 1) & 1, abort_flag, status);
-  } else if (warp == 1 && lane == 0 && n_iter > 0) {
+  } else if (warp == 1 && n_iter > 0) {
     // =========================== MMA issuer ===========================
+    // The whole warp walks the schedule in step, so that addresses and descriptors are the same in
+    // every lane; one elected lane (always the same one) issues the tensor-core instructions.
+    auto mwait = [&](uint32_t bar, uint32_t parity) -> bool {
+      return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, status));
+    };
     // S^T = K Q^T: A = K tile (K-major), B = Q (K-major).  O^T += V^T P^T: A = V tile transposed
     // (MN-major), B = P^T (MN-major).  Q K^T runs one tile ahead of the PV product, so the tensor
     // pipe has the scores of tile t+1 ready while the softmax of tile t is in flight.  The
@@ -247,8 +252,8 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
     auto issue_qk = [&]() -> bool {
       walk_tile(a, wq);
       const int it = wq.it, qb = wq.piece_idx & 1;
-      if ((wq.first && !mbar_wait(bars + 8 * (kTbQFull + qb), (wq.piece_idx >> 1) & 1, abort_flag, status)) ||
-          !mbar_wait(bars + 8 * (kTbKvFull + rk.buf), rk.par, abort_flag, status))
+      if ((wq.first && !mwait(bars + 8 * (kTbQFull + qb), (wq.piece_idx >> 1) & 1)) ||
+          !mwait(bars + 8 * (kTbKvFull + rk.buf), rk.par))
         return false;
       tc_fence_after();
       const uint32_t q_lo = q_lo0 + qb * (lay.q_bytes >> 4);
@@ -256,11 +261,11 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
       const uint32_t d_s = tmem + (it & 1) * NP;
 #pragma unroll
       for (int ks = 0; ks < KSTEPS_QK; ++ks)
-        umma_bf16_lo(d_s, k_lo + (ks >> 2) * (kHalfStrideT >> 4) + (ks & 3) * 2,
+        umma_bf16_lo_elect(d_s, k_lo + (ks >> 2) * (kHalfStrideT >> 4) + (ks & 3) * 2,
                      q_lo + (ks >> 2) * (NP * 128 >> 4) + (ks & 3) * 2, idesc_qk, ks > 0);
-      umma_commit(bars + 8 * (kTbKvEmpty + rk.buf));
-      umma_commit(bars + 8 * (kTbSFull + (it & 1)));
-      if (wq.last) umma_commit(bars + 8 * (kTbQEmpty + qb));
+      umma_commit_elect(bars + 8 * (kTbKvEmpty + rk.buf));
+      umma_commit_elect(bars + 8 * (kTbSFull + (it & 1)));
+      if (wq.last) umma_commit_elect(bars + 8 * (kTbQEmpty + qb));
       rk.step(2);
       walk_next(a, wq);
       return true;
@@ -277,22 +282,22 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
         int it = wp.it;
         for (; n_run > 0; --n_run, ++it) {
           // S^T(it + 1)
-          if (!mbar_wait(bars + 8 * (kTbKvFull + rk.buf), rk.par, abort_flag, status)) { ok = false; break; }
+          if (!mwait(bars + 8 * (kTbKvFull + rk.buf), rk.par)) { ok = false; break; }
           tc_fence_after();
           {
             const uint32_t k_lo = k_lo0 + rk.buf * (kKvBytes >> 4);
             const uint32_t d_s = tmem + ((it + 1) & 1) * NP;
 #pragma unroll
             for (int ks = 0; ks < KSTEPS_QK; ++ks)
-              umma_bf16_lo(d_s, k_lo + (ks >> 2) * (kHalfStrideT >> 4) + (ks & 3) * 2,
+              umma_bf16_lo_elect(d_s, k_lo + (ks >> 2) * (kHalfStrideT >> 4) + (ks & 3) * 2,
                            q_lo + (ks >> 2) * (NP * 128 >> 4) + (ks & 3) * 2, idesc_qk, ks > 0);
-            umma_commit(bars + 8 * (kTbKvEmpty + rk.buf));
-            umma_commit(bars + 8 * (kTbSFull + ((it + 1) & 1)));
+            umma_commit_elect(bars + 8 * (kTbKvEmpty + rk.buf));
+            umma_commit_elect(bars + 8 * (kTbSFull + ((it + 1) & 1)));
             rk.step(2);
           }
           // O^T += V^T P^T (it)
-          if (!mbar_wait(bars + 8 * (kTbPFull + (it & 1)), (it >> 1) & 1, abort_flag, status) ||
-              !mbar_wait(bars + 8 * (kTbKvFull + rv.buf), rv.par, abort_flag, status)) {
+          if (!mwait(bars + 8 * (kTbPFull + (it & 1)), (it >> 1) & 1) ||
+              !mwait(bars + 8 * (kTbKvFull + rv.buf), rv.par)) {
             ok = false;
             break;
           }
@@ -302,9 +307,9 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
             const uint32_t v_lo = v_lo0 + rv.buf * (kKvBytes >> 4);
 #pragma unroll
             for (int j = 0; j < kTile / 16; ++j)
-              umma_bf16_lo(tmem + kColO, v_lo + j * (2048 >> 4), p_lo + j * (2048 >> 4), idesc_pv, 1u);
-            umma_commit(bars + 8 * (kTbKvEmpty + rv.buf));
-            umma_commit(bars + 8 * (kTbPvDone + (it & 1)));
+              umma_bf16_lo_elect(tmem + kColO, v_lo + j * (2048 >> 4), p_lo + j * (2048 >> 4), idesc_pv, 1u);
+            umma_commit_elect(bars + 8 * (kTbKvEmpty + rv.buf));
+            umma_commit_elect(bars + 8 * (kTbPvDone + (it & 1)));
             rv.step(2);
           }
         }
@@ -318,8 +323,8 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
       if (wq.it < n_iter && !issue_qk()) { ok = false; break; }
       walk_tile(a, wp);
       const int it = wp.it;
-      if (!mbar_wait(bars + 8 * (kTbPFull + (it & 1)), (it >> 1) & 1, abort_flag, status) ||
-          !mbar_wait(bars + 8 * (kTbKvFull + rv.buf), rv.par, abort_flag, status)) {
+      if (!mwait(bars + 8 * (kTbPFull + (it & 1)), (it >> 1) & 1) ||
+          !mwait(bars + 8 * (kTbKvFull + rv.buf), rv.par)) {
         ok = false;
         break;
       }
@@ -331,20 +336,20 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
       if (ksteps == kTile / 16) {
 #pragma unroll
         for (int j = 0; j < kTile / 16; ++j)
-          umma_bf16_lo(tmem + kColO, v_lo + j * (2048 >> 4), p_lo + j * (2048 >> 4), idesc_pv, j == 0 ? acc0 : 1u);
+          umma_bf16_lo_elect(tmem + kColO, v_lo + j * (2048 >> 4), p_lo + j * (2048 >> 4), idesc_pv, j == 0 ? acc0 : 1u);
       } else {
 #pragma unroll 1
         for (int j = 0; j < ksteps; ++j)
-          umma_bf16_lo(tmem + kColO, v_lo + j * (2048 >> 4), p_lo + j * (2048 >> 4), idesc_pv, j == 0 ? acc0 : 1u);
+          umma_bf16_lo_elect(tmem + kColO, v_lo + j * (2048 >> 4), p_lo + j * (2048 >> 4), idesc_pv, j == 0 ? acc0 : 1u);
       }
-      umma_commit(bars + 8 * (kTbKvEmpty + rv.buf));
-      umma_commit(bars + 8 * (kTbPvDone + (it & 1)));
+      umma_commit_elect(bars + 8 * (kTbKvEmpty + rv.buf));
+      umma_commit_elect(bars + 8 * (kTbPvDone + (it & 1)));
       rv.step(2);
       walk_next(a, wp);
     }
     if (!ok) {
       // aborting: let the tensor pipe run dry before tensor memory is released
-      umma_commit(bars + 8 * kTbDrain);
+      umma_commit_elect(bars + 8 * kTbDrain);
       const unsigned long long t_begin = global_ns();
       while (!mbar_try_wait(bars + 8 * kTbDrain, 0) && global_ns() - t_begin < wait_limit_ns(abort_flag)) {
       }
