@@ -43,8 +43,8 @@ UNIT = "tokens/s"
 METRIC_CONFIG = "step query tokens/s (Predict+Verify step of the named configuration: RoPE, attention, accept, append, all layers)"
 SEG_LEN, MEM_TOKENS = 512, 170          # one compaction: 512-token step -> 170 memory tokens + <o>
 FALLBACK_HBM_GBS = 6650.0
-# DRAM bytes the split kernel moved per algorithmic byte in an ncu capture of the batch-32 point
-# of the same workload (scaled by the bytes streamed).
+# DRAM bytes the split kernel moved per algorithmic byte in an ncu capture of the batch-48 point
+# of the same workload (scaled by the bytes streamed); taken with the kernel as it stands.
 NCU_TRAFFIC_PER_ALGO_BYTE = 1.011
 KERNELS_PER_STEP = 5                    # rope, attention (merge in its tail), accept, append, compaction
 
