@@ -69,7 +69,7 @@ def gpu_attn(P, sm_scale=0.0, want_lse=True, canary=True, device="cuda", ws_min_
     out = out_buf[pad:pad + T * Hq * D].view(T, Hq, D)
     lse_buf = torch.full((max(T, 1) * Hq + 2 * pad,), 7.0, dtype=torch.float32, device=dev)
     lse = lse_buf[pad:pad + T * Hq].view(T, Hq)
-    max_kv = max(P["lens"] + [0])
+    max_kv = max(P["lens"] + [0, P.get("max_kv_len", 0)])      # the host's bound may exceed every actual length
     ws_bytes = ms.memosight_attn_workspace_bytes(P["B"], Hq, P["Hkv"], D, max_kv, P["max_nq"])
     assert ws_bytes > 0
     ws_bytes = max(ws_bytes, ws_min_bytes)

@@ -123,3 +123,32 @@ def test_rows_that_see_nothing_at_first_and_only_strongly_negative_scores_later(
             assert torch.equal(out[i, kvh * 4], P["v_step"][i, kvh]), "a single visible key: the output is its V row"
             assert abs(float(lse[i, kvh * 4]) + 150.0) < 1.0
     assert bool(torch.isfinite(out.float()).all())
+
+
+def test_chunk_without_a_visible_key_beside_a_chunk_of_strongly_negative_scores():
+    # The same rows, but the host's bound on the cache length is far above the (empty) cache, so the
+    # launch cuts every unit into chunks and the two or three key tiles of a unit land in different
+    # chunks.  A foresight row with anchor 0 then sees nothing at all in the chunk that holds the
+    # block's first key tile and one key, 150 nats below zero, in a later chunk: the empty chunk's
+    # partial must not take part in the merge (were it to carry a reference of 0, the real chunk's
+    # weight 2^-216 would flush to zero and the row would come out as 0/0).
+    P = random_problem(1, 8, 2, 128, [0], [300], [120], seed=62, anchors=True)
+    P["max_kv_len"] = 30000
+    rows = [130, 201, 299]
+    for i in rows:
+        P["anchor"][i] = 0
+        for kvh in range(2):
+            q = P["q"][i, kvh * 4].float()
+            P["k_step"][i, kvh] = (-150.0 * np.sqrt(128) * q / q.norm() ** 2).to(torch.bfloat16)
+    out, lse = check_attn(P, "chunked unit, an empty chunk beside strongly negative scores")
+    for i in rows:
+        for kvh in range(2):
+            assert torch.equal(out[i, kvh * 4], P["v_step"][i, kvh])
+            assert abs(float(lse[i, kvh * 4]) + 150.0) < 1.0
+    assert bool(torch.isfinite(out.float()).all())
+    # and a plain chunked block with short tiles in the right half of a tile only: the second
+    # accumulator of an item may stay unwritten (every tile of the item has at most 64 valid keys)
+    Q = random_problem(2, 8, 2, 128, [40, 64], [70, 100], [70, 100], seed=63)
+    Q["max_kv_len"] = 30000
+    check_attn(Q, "chunked units whose tiles hold at most 64 keys")
+    check_attn(random_problem(2, 8, 2, 128, [40, 64], [40, 64], [40, 64], seed=64), "whole units of at most 64 keys per tile")
