@@ -371,6 +371,7 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
     Walk w = w0;
     float lsum[CW];
     uint32_t wg_phase = 0;
+    int plain_left = 0;        // plain tiles ahead in the current run (used where the tile body exists once)
     bool ok = true;
     auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {
       return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, status));
@@ -529,16 +530,26 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
         }
         if (!ok) break;
       }
-      walk_tile(a, w);
+      // Without the separate loop above, a plain tile at least skips the schedule walker: the same
+      // tile body runs with the facts of a full cache tile in the middle of its piece.
+      bool plain = false;
+      if (!kPlainSoftmax) {
+        if (plain_left <= 0 && w.open) plain_left = min(w.L / kTile - w.ti, n_iter - 1 - w.it);
+        plain = plain_left > 0;
+      }
+      if (!plain) walk_tile(a, w);
       const int it = w.it, pb = it & 1;
       if (!wait_all(bars + 8 * (kTbSFull + pb), (it >> 1) & 1)) { ok = false; break; }
       tc_fence_after();
-      const int nv = w.nvalid;
+      const int nv = plain ? kTile : w.nvalid;
+      const bool is_step = plain ? false : w.is_step;
+      const bool opens = plain ? false : (w.piece_j == 0);
+      const bool closes = plain ? false : w.last;
       const uint32_t s_addr = lane_addr + pb * NP + c0;
       float v[CW];
-      load_scores(v, s_addr, nv, w.is_step);
+      load_scores(v, s_addr, nv, is_step);
 
-      if (w.piece_j == 0) {
+      if (opens) {
         // new unit: the reference maximum of each row is the exact maximum of this first tile
         reduce_row_max(v);
         if (!wg_sync()) { ok = false; break; }
@@ -552,15 +563,15 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
       }
 
       const float tmaxx = shift_scores(v);
-      if (w.piece_j > 0) {
+      if (!opens) {
         // the four warps agree on whether any score outgrew its reference (tile index as the token);
         // a piece's first tile set the references from its own scores and cannot outgrow them
         if (__any_sync(0xffffffffu, tmaxx > kGrowLimit) && lane == 0) *grow_flag = it + 1;
         if (!wg_sync()) { ok = false; break; }
-        if (*grow_flag == it + 1 && !regrow(v, it, s_addr, nv, w.is_step)) { ok = false; break; }
+        if (*grow_flag == it + 1 && !regrow(v, it, s_addr, nv, is_step)) { ok = false; break; }
       }
       emit_p(v, pb);
-      if (w.is_step || nv < kTile) {
+      if (is_step || nv < kTile) {
         // V rows past the valid keys hold foreign or stale bytes; their P is 0 but 0 * NaN is NaN:
         // clear the rows of the last 16-key step that the PV product still reads.  Done behind the
         // exponentials, so that the wait for the V tile (which lands after the K tile) overlaps them,
@@ -576,8 +587,15 @@ attn_umma_t_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k,
         }
       }
       publish_p(pb);
+      if (plain) {
+        ++w.ti;
+        ++w.it;
+        ++w.piece_j;
+        --plain_left;
+        continue;
+      }
 
-      if (w.last) {
+      if (closes) {
         // ---- end of the unit (or of this CTA's part of it) ----
         // row sums: over the 32 lanes of each warp, then over the four warps
         {
