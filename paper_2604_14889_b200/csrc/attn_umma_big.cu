@@ -540,6 +540,7 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
     bool o1_live = false;   // the second accumulator has been written in this item (a tile with more than 64 valid keys)
     int tok = 0, anc = 0, rows = 0;
     bool row_ok = false;
+    bool warp_live = true;    // some row of this warp's 32 exists in the item's row tile
     uint32_t all_phase = 0;
     bool ok = true;
     auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {
@@ -580,6 +581,24 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
           const uint32_t addr = va + (cc >> 3) * kBHalf + rr * 128 + ((cc & 7) << 4);
           asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(addr), "r"(0u) : "memory");
         }
+      }
+      if (!warp_live) {
+        // A warp whose 32 rows all lie past the end of a short last row tile (44 of 128 rows in the
+        // last tile of a 171-token block at G = 4) has nothing to exponentiate: what its rows of P
+        // and O hold is never stored, and rows do not mix.  It only keeps in step -- it has waited
+        // for the scores like the others and arrives like them -- and leaves the special-function
+        // unit to the warps that have rows.
+        if (opens_item) {
+          unref = true;
+          l_part = 0.f;
+          o1_live = false;
+        }
+        if (nv > kBCw) o1_live = true;
+        if (masked && (nv & 15)) fence_async_smem();
+        tc_fence_before();
+        __syncwarp();
+        mbar_arrive_if(lane == 0, bars + 8 * (kBbPFull + pb));
+        return true;
       }
       // this warpgroup's score columns of the row; invisible keys become -inf
       const uint32_t s_addr = lane_addr + kBColS + pb * kTile + wg * kBCw;
@@ -705,6 +724,7 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
         const int tok0 = w.rt * tpt;
         rows = (min(w.s.n_q, tok0 + tpt) - tok0) * a.G;
         row_ok = r < rows;
+        warp_live = quad * 32 < rows;
         if (row_ok) {
           const int i = tok0 + r / a.G;
           tok = i;
@@ -742,7 +762,7 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
         const float inv = (w.slot < 0) ? 1.f / l_row : 1.f;     // a partial stays unnormalised, relative to m_row
         const float f0 = w0 * inv, f1 = w1 * inv;
 #pragma unroll 1
-        for (int c = 0; c < kBCw / 32; ++c) {
+        for (int c = 0; c < (warp_live ? kBCw / 32 : 0); ++c) {
           uint32_t o[32];
           tmem_ld32(lane_addr + kBColO + wg * kBCw + c * 32, o);
           tmem_ld_wait(o);
