@@ -66,7 +66,8 @@ static_assert(kBbCount * 8 <= kBMiscScalars, "barriers overflow their slot");
 // tiles need is fetched from HBM once and found in L2 by the others.  A unit's tiles (cache tiles,
 // then the step-local key tiles up to the row tile's last token) are cut into `nsplit` chunks only
 // when there are too few units to fill the machine; a chunked unit leaves one (m, l, O) partial per
-// chunk for attn_big_merge_kernel.
+// chunk for attn_big_merge_kernel.  With more units than CTAs only the units of the last, partial
+// round are cut (big_tail below).
 
 struct BigSeq {
   int L, n_q, r0, n_c, cache_tiles, n_rt;
@@ -111,10 +112,29 @@ attn_big_plan_kernel(const AttnArgs a, int tpt, int* __restrict__ pre) {
   if (tid == nt - 1) pre[a.B] = base;
 }
 
+// Whole units dealt round-robin leave the last round ragged: 512 units on 148 CTAs are three full
+// rounds and 68 units more, and the launch lasts four units while the average CTA has 3.46.  When
+// units are not chunked anyway, the units of that last, partial round are cut into `split` chunks
+// each (as many as fit the grid once more), so that the round costs 1 / split of a unit: units
+// [0, u0) stay whole, unit u0 + t / split, chunk t % split is item u0 + t, and its partial goes to
+// slot t (at most one per CTA) for attn_big_tail_merge_kernel.  Both kernels derive (u0, split)
+// from the unit count with this function.
+constexpr int kBMaxTailSplit = 8;
+__device__ __forceinline__ void big_tail(int units, int n_ctas, int nsplit, int& u0, int& split) {
+  u0 = units;
+  split = 1;
+  if (nsplit != 1 || units <= n_ctas) return;
+  const int rem = units % n_ctas;
+  if (rem == 0 || n_ctas / rem < 2) return;
+  split = min(n_ctas / rem, kBMaxTailSplit);
+  u0 = units - rem;
+}
+
 struct BigWalk {
   BigSeq s;
   int b, h, rt, ti, ti_lo, ti_hi, tpt;
   int item, n_items, nsplit;
+  int tail_u0, tail_split, item_slot;
   int it, piece_idx, piece_j, slot;
   bool first, last, done;
   int step_idx, nvalid;     // step_idx < 0: cache tile
@@ -124,24 +144,37 @@ __device__ __forceinline__ void bwalk_advance(const AttnArgs& a, BigWalk& w, con
   for (;;) {
     w.item += static_cast<int>(gridDim.x);
     if (w.item >= w.n_items) { w.done = true; return; }
+    // index in the (sequence, head, chunk, row tile) order; a unit of the cut last round comes with its own chunk
+    int idx = w.item, tail_chunk = -1;
+    if (w.item >= w.tail_u0) {
+      const int t = w.item - w.tail_u0;
+      idx = w.tail_u0 + t / w.tail_split;
+      tail_chunk = t - (t / w.tail_split) * w.tail_split;
+    }
     const int per_rt = a.H_kv * w.nsplit;                 // items per row tile of a sequence
     int lo = 0, hi = a.B;
     while (hi - lo > 1) {
       const int mid = (lo + hi) >> 1;
-      if (static_cast<long long>(pre[mid]) * per_rt <= w.item) lo = mid; else hi = mid;
+      if (static_cast<long long>(pre[mid]) * per_rt <= idx) lo = mid; else hi = mid;
     }
     w.b = lo;
     big_seq(a, lo, w.tpt, w.s);
     if (w.s.n_rt == 0) continue;                          // cannot happen for a valid index; stay safe
-    int j = w.item - pre[lo] * per_rt;
+    int j = idx - pre[lo] * per_rt;
     const int per_head = w.nsplit * w.s.n_rt;
     w.h = j / per_head;
     j -= w.h * per_head;
-    const int chunk = j / w.s.n_rt;
+    int chunk = j / w.s.n_rt, n_chunks = w.nsplit;
     w.rt = j - chunk * w.s.n_rt;
+    w.item_slot = (w.nsplit == 1) ? -1 : w.item;
+    if (tail_chunk >= 0) {
+      chunk = tail_chunk;
+      n_chunks = w.tail_split;
+      w.item_slot = w.item - w.tail_u0;
+    }
     const int tiles_u = w.s.cache_tiles + big_step_tiles(w.s, w.rt, w.tpt);
-    w.ti_lo = static_cast<int>(static_cast<long long>(tiles_u) * chunk / w.nsplit);
-    w.ti_hi = static_cast<int>(static_cast<long long>(tiles_u) * (chunk + 1) / w.nsplit);
+    w.ti_lo = static_cast<int>(static_cast<long long>(tiles_u) * chunk / n_chunks);
+    w.ti_hi = static_cast<int>(static_cast<long long>(tiles_u) * (chunk + 1) / n_chunks);
     if (w.ti_lo < w.ti_hi) break;
   }
   w.ti = w.ti_lo;
@@ -149,7 +182,13 @@ __device__ __forceinline__ void bwalk_advance(const AttnArgs& a, BigWalk& w, con
 __device__ __forceinline__ void bwalk_init(const AttnArgs& a, BigWalk& w, int tpt, int nsplit, const int* pre) {
   w.tpt = tpt;
   w.nsplit = nsplit;
-  w.n_items = pre[a.B] * a.H_kv * nsplit;
+  {
+    const int units = pre[a.B] * a.H_kv;
+    big_tail(units, static_cast<int>(gridDim.x), nsplit, w.tail_u0, w.tail_split);
+    w.n_items = (nsplit == 1) ? w.tail_u0 + (units - w.tail_u0) * w.tail_split : units * nsplit;
+    if (nsplit != 1) w.tail_u0 = w.n_items;             // no item is a tail item
+  }
+  w.item_slot = -1;
   w.item = static_cast<int>(blockIdx.x) - static_cast<int>(gridDim.x);
   w.it = 0;
   w.piece_idx = -1;
@@ -161,7 +200,7 @@ __device__ __forceinline__ void bwalk_init(const AttnArgs& a, BigWalk& w, int tp
 __device__ __forceinline__ void bwalk_tile(BigWalk& w) {
   w.first = (w.ti == w.ti_lo);
   if (w.first) {
-    w.slot = (w.nsplit == 1) ? -1 : w.item;
+    w.slot = w.item_slot;
     w.piece_idx += 1;
     w.piece_j = 0;
   }
@@ -819,43 +858,32 @@ attn_umma_big_kernel(const AttnArgs a, const __grid_constant__ CUtensorMap map_k
   }
 }
 
-// One CTA per (sequence, KV head, row tile) unit of a chunked launch; one warp per packed row
-// folds the chunks' (m, l) with shuffles and accumulates its output columns.
-__global__ void __launch_bounds__(128)
-attn_big_merge_kernel(const AttnArgs a, int tpt, int max_rt, int nsplit) {
+// The partials of one (sequence, KV head, row tile) unit folded into its output rows; one warp per
+// packed row folds the chunks' (m, l) with shuffles and accumulates its output columns.  Chunk k's
+// partial is slot slot0 + k * slot_stride; a chunk without tiles has none.
+__device__ __forceinline__ void big_merge_unit(const AttnArgs& a, const BigSeq& s, int h, int rt, int tpt, int n_chunks,
+                                               long long slot0, long long slot_stride,
+                                               const float* __restrict__ ws_slots) {
   constexpr int D = kBD, E = D / 32;
-  int u = blockIdx.x;
-  const int rt = u % max_rt; u /= max_rt;
-  const int h = u % a.H_kv;
-  const int b = u / a.H_kv;
-  const int* pre = reinterpret_cast<const int*>(reinterpret_cast<const uint8_t*>(a.workspace) + kWsHeaderBytes);
-  const float* ws_slots = reinterpret_cast<const float*>(
-      reinterpret_cast<const uint8_t*>(a.workspace) + kWsHeaderBytes + ws_prefix_bytes());
-  BigSeq s;
-  big_seq(a, b, tpt, s);
-  if (rt >= s.n_rt) return;
   const int tiles_u = s.cache_tiles + big_step_tiles(s, rt, tpt);
-  // slot of chunk k = its item index; a chunk without tiles has no partial
-  const long long item0 = static_cast<long long>(pre[b]) * a.H_kv * nsplit +
-                          static_cast<long long>(h) * nsplit * s.n_rt + rt;
   const int tok0 = rt * tpt;
   const int rows = (min(s.n_q, tok0 + tpt) - tok0) * a.G;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const size_t slot_floats = big_slot_floats();
   for (int r = warp; r < rows; r += 4) {
     float M = -INFINITY;
-    if (lane < nsplit) {
-      const bool has = static_cast<long long>(tiles_u) * lane / nsplit < static_cast<long long>(tiles_u) * (lane + 1) / nsplit;
-      if (has) M = ws_slots[(item0 + static_cast<long long>(lane) * s.n_rt) * slot_floats + static_cast<size_t>(kTile) * D + r];
+    if (lane < n_chunks) {
+      const bool has = static_cast<long long>(tiles_u) * lane / n_chunks < static_cast<long long>(tiles_u) * (lane + 1) / n_chunks;
+      if (has) M = ws_slots[(slot0 + static_cast<long long>(lane) * slot_stride) * slot_floats + static_cast<size_t>(kTile) * D + r];
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
     float Lsum = 0.f, acc[E];
 #pragma unroll
     for (int e = 0; e < E; ++e) acc[e] = 0.f;
-    for (int k = 0; k < nsplit; ++k) {
-      if (static_cast<long long>(tiles_u) * k / nsplit >= static_cast<long long>(tiles_u) * (k + 1) / nsplit) continue;
-      const float* sp = ws_slots + (item0 + static_cast<long long>(k) * s.n_rt) * slot_floats;
+    for (int k = 0; k < n_chunks; ++k) {
+      if (static_cast<long long>(tiles_u) * k / n_chunks >= static_cast<long long>(tiles_u) * (k + 1) / n_chunks) continue;
+      const float* sp = ws_slots + (slot0 + static_cast<long long>(k) * slot_stride) * slot_floats;
       const float m = sp[static_cast<size_t>(kTile) * D + r];
       const float l = sp[static_cast<size_t>(kTile) * D + kTile + r];
       const float wgt = (m == -INFINITY) ? 0.f : exp2f(m - M);
@@ -872,6 +900,50 @@ attn_big_merge_kernel(const AttnArgs a, int tpt, int max_rt, int nsplit) {
     for (int e = 0; e < E; e += 2) *reinterpret_cast<uint32_t*>(op + e) = pack2(acc[e] * inv, acc[e + 1] * inv);
     if (a.lse && lane == 0) a.lse[orow] = (M + log2f(Lsum)) * 0.69314718055994531f;
   }
+}
+
+// One CTA per (sequence, KV head, row tile) unit of a chunked launch.
+__global__ void __launch_bounds__(128)
+attn_big_merge_kernel(const AttnArgs a, int tpt, int max_rt, int nsplit) {
+  int u = blockIdx.x;
+  const int rt = u % max_rt; u /= max_rt;
+  const int h = u % a.H_kv;
+  const int b = u / a.H_kv;
+  const int* pre = reinterpret_cast<const int*>(reinterpret_cast<const uint8_t*>(a.workspace) + kWsHeaderBytes);
+  const float* ws_slots = reinterpret_cast<const float*>(
+      reinterpret_cast<const uint8_t*>(a.workspace) + kWsHeaderBytes + ws_prefix_bytes());
+  BigSeq s;
+  big_seq(a, b, tpt, s);
+  if (rt >= s.n_rt) return;
+  // slot of chunk k = its item index
+  const long long item0 = static_cast<long long>(pre[b]) * a.H_kv * nsplit +
+                          static_cast<long long>(h) * nsplit * s.n_rt + rt;
+  big_merge_unit(a, s, h, rt, tpt, nsplit, item0, s.n_rt, ws_slots);
+}
+
+// One CTA per unit of the cut last round of an unchunked launch (see big_tail); n_ctas is the grid
+// of the attention kernel that wrote the partials.
+__global__ void __launch_bounds__(128)
+attn_big_tail_merge_kernel(const AttnArgs a, int tpt, int n_ctas) {
+  const int* pre = reinterpret_cast<const int*>(reinterpret_cast<const uint8_t*>(a.workspace) + kWsHeaderBytes);
+  const float* ws_slots = reinterpret_cast<const float*>(
+      reinterpret_cast<const uint8_t*>(a.workspace) + kWsHeaderBytes + ws_prefix_bytes());
+  const int units = pre[a.B] * a.H_kv;
+  int u0, split;
+  big_tail(units, n_ctas, 1, u0, split);
+  const int u = u0 + static_cast<int>(blockIdx.x);
+  if (split == 1 || u >= units) return;
+  int lo = 0, hi = a.B;
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (static_cast<long long>(pre[mid]) * a.H_kv <= u) lo = mid; else hi = mid;
+  }
+  BigSeq s;
+  big_seq(a, lo, tpt, s);
+  if (s.n_rt == 0) return;
+  const int j = u - pre[lo] * a.H_kv;
+  const int h = j / s.n_rt, rt = j - h * s.n_rt;
+  big_merge_unit(a, s, h, rt, tpt, split, static_cast<long long>(blockIdx.x) * split, 1, ws_slots);
 }
 
 // Chunks per unit, from a small cost model in units of one tile's time: items are dealt
@@ -897,7 +969,7 @@ int big_nsplit(int B, int H_kv, int max_rt, int n_ctas, int max_kv_len) {
 }  // namespace
 
 // Large blocks, and step blocks with more than 64 packed rows (where two softmax warpgroups per
-// tile beat the one of the rows-on-lanes step kernel: 5.2 against 4.2 TB/s at 128 rows).
+// tile beat the one of the rows-on-lanes step kernel: 5.9 against 4.2 TB/s at 128 rows).
 bool attn_umma_big_supports(int D, int G, int max_nq) {
   return D == kBD && G >= 1 && G <= kMaxGroup && max_nq <= kMaxNqBig && (max_nq > kMaxNq || G * max_nq > 64);
 }
@@ -905,7 +977,8 @@ bool attn_umma_big_supports(int D, int G, int max_nq) {
 size_t attn_umma_big_workspace_bytes(int B, int H_kv, int G, int max_nq, int max_kv_len, int n_ctas) {
   const int tpt = kTile / G, max_rt = (max_nq + tpt - 1) / tpt;
   const int nsplit = big_nsplit(B, H_kv, max_rt, n_ctas, max_kv_len);
-  const size_t slots = nsplit > 1 ? static_cast<size_t>(B) * H_kv * max_rt * nsplit : 0;
+  // chunked launch: one partial per item; otherwise at most one per CTA for the cut last round
+  const size_t slots = nsplit > 1 ? static_cast<size_t>(B) * H_kv * max_rt * nsplit : static_cast<size_t>(n_ctas);
   return kWsHeaderBytes + ws_prefix_bytes() + slots * big_slot_floats() * sizeof(float);
 }
 
@@ -943,6 +1016,11 @@ int32_t launch_attn_umma_big(const AttnArgs& a, cudaStream_t st) {
   if (nsplit > 1) {
     const long long units = static_cast<long long>(a.B) * a.H_kv * max_rt;
     attn_big_merge_kernel<<<static_cast<unsigned>(units), 128, 0, st>>>(a, tpt, max_rt, nsplit);
+    MS_LAUNCH_CHECK();
+  } else if (static_cast<long long>(a.B) * a.H_kv * max_rt > grid) {
+    // more units than CTAs are possible: the last round may have been cut (the kernel decides from
+    // the actual block sizes; CTAs of this grid beyond the cut units return at once)
+    attn_big_tail_merge_kernel<<<grid, 128, 0, st>>>(a, tpt, grid);
     MS_LAUNCH_CHECK();
   }
   return MS_OK;

@@ -152,3 +152,19 @@ def test_chunk_without_a_visible_key_beside_a_chunk_of_strongly_negative_scores(
     Q["max_kv_len"] = 30000
     check_attn(Q, "chunked units whose tiles hold at most 64 keys")
     check_attn(random_problem(2, 8, 2, 128, [40, 64], [40, 64], [40, 64], seed=64), "whole units of at most 64 keys per tile")
+
+
+def test_more_units_than_ctas_cut_their_last_round():
+    # 40 sequences x 2 KV heads x 2 row tiles = 160 units on 148 CTAs (fewer on a smaller part: the
+    # case then still runs, uncut): the 12 units of the last round are cut into chunks, each leaves a
+    # partial, and a second kernel merges them.  Ragged caches, so the chunks differ in length; a few
+    # short blocks (one row tile) shift the unit numbering.
+    rng = np.random.default_rng(71)
+    lens = [int(x) for x in rng.integers(900, 3000, size=40)]
+    n_q = [40] * 40
+    n_q[3], n_q[17], n_q[39] = 33, 48, 64
+    P = random_problem(40, 8, 2, 128, lens, n_q, n_q, seed=72)
+    check_attn(P, "160 units: the last round cut into chunks")
+    # and with foresight rows and custom anchors in the cut units
+    Q = random_problem(40, 8, 2, 128, lens, n_q, [30] * 40, seed=73, anchors=True)
+    check_attn(Q, "160 units, custom anchors")
