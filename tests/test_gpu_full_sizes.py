@@ -35,14 +35,15 @@ def _attn_all(inp, layer=0, q=None, ks=None):
     return out, lse
 
 
-def _check_sampled_units(inp, out, lse, n_samples, seed, layer=0):
-    """Oracle on single (sequence, KV head) units cut out of the device tensors."""
+def _check_sampled_units(inp, out, lse, n_samples, seed, layer=0, units=None):
+    """Oracle on single (sequence, KV head) units cut out of the device tensors (`units`: explicit
+    (sequence, KV head) pairs instead of hashed ones)."""
     c = inp.cfg
     G, D, nq = c.group, c.head_dim, c.n_q
     worst, peak_ref = 0.0, 0.0
-    for i in range(n_samples):
+    for i in range(n_samples if units is None else len(units)):
         h = synth.hash_scalar(i, seed, 99)
-        b, kvh = h % c.batch, (h >> 20) % c.n_kv_heads
+        b, kvh = (h % c.batch, (h >> 20) % c.n_kv_heads) if units is None else units[i]
         L, o = inp.lens[b], inp.offs[b]
         kc = bits(inp.k_cache[layer, kvh, o:o + L])[None]
         vc = bits(inp.v_cache[layer, kvh, o:o + L])[None]
@@ -136,3 +137,26 @@ def test_long_cot_config_two_physical_layers_attention_and_compaction():
         got = bits((inp.k_cache if is_k else inp.v_cache)[layer, kvh, inp.offs[b]:inp.offs[b] + L - 512])
         assert np.array_equal(got, k1[0, 0, :L - 512])
         assert np.array_equal(src[b, :L - 512].cpu().numpy(), want_src[0, :L - 512])
+
+
+def test_compression_event_batch64_sampled_units():
+    # the secondary benchmark's launch: 64 sequences, cache 16 384 + the 512-token step, a causal
+    # block of 170 memory tokens + <o> per sequence (six row tiles per KV head, the last one 44 rows)
+    cfg = synth.StepConfig("compress-full", 64, 32, 8, 128, 16896, 16896, 171, 0, 5.0e5, 1024, seed=0x5EED0004)
+    inp = synth.make_step_inputs(cfg, device=DEV)
+    out, lse = _attn_all(inp)
+    out2, lse2 = _attn_all(inp)
+    assert torch.equal(out, out2) and torch.equal(lse, lse2)
+    assert bool(torch.isfinite(out.float()).all())
+    _check_sampled_units(inp, out, lse, 3, seed=5)
+
+
+def test_wide_group_step_blocks_batch128_units_of_the_cut_last_round():
+    # G = 8, 12-token blocks (96 packed rows) at batch 128: 512 units for the large-block kernel;
+    # on 148 CTAs units 444..511 (sequences 111..127) are the ones cut into chunks and merged
+    cfg = synth.StepConfig("g8-full", 128, 32, 4, 128, 16384, 16384, 6, 6, 5.0e5, 1024, seed=0x5EED0006)
+    inp = synth.make_step_inputs(cfg, device=DEV)
+    out, lse = _attn_all(inp)
+    out2, lse2 = _attn_all(inp)
+    assert torch.equal(out, out2) and torch.equal(lse, lse2)
+    _check_sampled_units(inp, out, lse, 0, seed=6, units=[(0, 0), (57, 3), (110, 3), (111, 0), (119, 2), (127, 3)])
